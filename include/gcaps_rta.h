@@ -1,0 +1,186 @@
+/*
+ * gcaps_rta.h -- C ABI of the batched worst-case response-time analysis (RTA) library
+ * for GPU-using real-time tasksets (GCAPS, ECRTS 2024, arXiv 2406.05221).
+ *
+ * One call analyses n_tasksets independent tasksets on one NVIDIA B200 (sm_100a).  For every
+ * taskset it walks the tasks in decreasing priority and solves the integer fixed-point
+ * response-time recurrence of the paper's Sec. 6 (Eq. 1, Eq. 2, Eq. 4 with the lemma set of
+ * the chosen analysis), and writes one worst-case response time (WCRT) per task and one
+ * schedulable flag per taskset.
+ *
+ * All times are integer microseconds held as int64_t.  Nothing in this header is a torch type;
+ * device buffers are plain device pointers owned by the caller.
+ */
+#ifndef GCAPS_RTA_H_
+#define GCAPS_RTA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GCAPS_RTA_VERSION 100 /* major*100 + minor */
+
+/* ---- limits of the input domain ------------------------------------------------------------ */
+#define GCAPS_RTA_MAX_TASKS 256              /* tasks per taskset                                */
+#define GCAPS_RTA_MAX_SEGMENTS 65536         /* CPU segments, and GPU segments, per task         */
+#define GCAPS_RTA_MAX_TIME (1LL << 40)       /* every period, deadline, WCET, L and overhead     */
+#define GCAPS_RTA_MAX_CORE ((1LL << 31) - 1) /* CPU core ids are 0 .. MAX_CORE                   */
+#define GCAPS_RTA_ITER_CAP (1LL << 20)       /* fixed-point sweeps per task before ITER_LIMIT    */
+
+/* ---- policy argument ------------------------------------------------------------------------
+ * Low byte: the GPU arbitration policy that is analysed.
+ *   GCAPS_POLICY_GCAPS  preemptive priority-based GPU context scheduling (Sec. 6.3, Lemmas 8-15)
+ *   GCAPS_POLICY_RR     default work-conserving round-robin time-sliced driver (Sec. 6.2,
+ *                       Lemmas 1-7)
+ * OR-able flags:
+ *   GCAPS_RTA_BUSY      tasks busy-wait on the CPU during pure GPU execution (the "busy-waiting
+ *                       mode" lemmas); without it tasks self-suspend (the "self-suspension mode"
+ *                       lemmas).
+ *   GCAPS_RTA_LITERAL   evaluate the lemmas exactly as printed.  Without it two printed forms
+ *                       are repaired: (a) RR self-suspension, Lemma 7: the jitter J^c_h is taken
+ *                       as 0 for a CPU-only tau_h (a task without GPU segments never suspends);
+ *                       (b) GCAPS busy-waiting, Lemma 10: the busy-wait G^{e*}_h of a same-core
+ *                       GPU-using tau_h is charged to tau_i also when tau_i is CPU-only.
+ */
+#define GCAPS_POLICY_GCAPS 0
+#define GCAPS_POLICY_RR 1
+#define GCAPS_RTA_BUSY 0x100
+#define GCAPS_RTA_LITERAL 0x200
+
+/* ---- values written to out_sched[t] --------------------------------------------------------- */
+#define GCAPS_SCHED_NO 0      /* some task's bound exceeds its deadline (or hit ITER_LIMIT)      */
+#define GCAPS_SCHED_YES 1     /* every task converged to R_i <= D_i (an empty taskset is YES)    */
+#define GCAPS_SCHED_INVALID 2 /* the taskset is outside the input domain; nothing was analysed   */
+
+/* ---- sentinels written to out_wcrt[k] (all negative; a converged bound is >= 0) ------------- */
+#define GCAPS_WCRT_MISS (-1)       /* first task, in priority order, whose iterate exceeded D_i  */
+#define GCAPS_WCRT_SKIPPED (-2)    /* every task after the first MISS / ITER_LIMIT in that order */
+#define GCAPS_WCRT_ITER_LIMIT (-3) /* GCAPS_RTA_ITER_CAP sweeps without convergence or miss      */
+#define GCAPS_WCRT_INVALID (-4)    /* task of an INVALID taskset (when its slot is addressable)  */
+
+/* ---- return codes ---------------------------------------------------------------------------- */
+#define GCAPS_OK 0
+#define GCAPS_ERR_INVALID_ARG (-1)   /* null pointer, negative count, unknown policy bits, L<=0
+                                        for RR, overhead<0, a time argument above MAX_TIME      */
+#define GCAPS_ERR_WORKSPACE (-2)     /* workspace null or smaller than gcaps_rta_workspace_bytes */
+#define GCAPS_ERR_CUDA (-3)          /* a CUDA runtime call failed; see gcaps_rta_last_cuda_error */
+#define GCAPS_ERR_NO_DEVICE (-4)     /* no CUDA device / not an sm_100 device                    */
+
+/*
+ * A batch of tasksets in CSR structure-of-arrays form (task model: Sec. 4).
+ *
+ * Taskset t owns tasks task_off[t] .. task_off[t+1]-1 of the per-task arrays.  Task k owns CPU
+ * segments cseg_off[k] .. cseg_off[k+1]-1 (eta^c_k of them) and GPU segments gseg_off[k] ..
+ * gseg_off[k+1]-1 (eta^g_k of them; none for a CPU-only task).  GPU segment j of a task is the
+ * pair (G^m = gseg_misc[j], G^e = gseg_exec[j]): miscellaneous CPU work and pure GPU work.
+ * The task-level quantities of the paper are sums over the task's segments:
+ *   C_i = sum cseg_wcet,  G^m_i = sum gseg_misc,  G^e_i = sum gseg_exec,  G_i = G^m_i + G^e_i.
+ * A larger priority value means a higher priority; equal priorities are ordered by position
+ * (the earlier task is the higher one).  The order of tasks inside a taskset is free.
+ *
+ * Every pointer of one struct is either a device pointer (gcaps_rta_batch, gcaps_rta_validate)
+ * or a host pointer (gcaps_rta_batch_host).  The library only reads these arrays and keeps no
+ * pointer after the call's work has completed.
+ *
+ * Domain of a valid taskset: 0 <= n <= GCAPS_RTA_MAX_TASKS tasks; offsets non-decreasing and
+ * inside [0, n_tasks], [0, n_csegs], [0, n_gsegs]; at most GCAPS_RTA_MAX_SEGMENTS segments of a
+ * kind per task; 1 <= D_i <= T_i <= GCAPS_RTA_MAX_TIME; 0 <= core <= GCAPS_RTA_MAX_CORE; every
+ * segment WCET in [0, GCAPS_RTA_MAX_TIME].
+ */
+typedef struct gcaps_tasksets {
+  int64_t n_tasks;          /* length of the per-task arrays (= task_off[n_tasksets])            */
+  int64_t n_csegs;          /* length of cseg_wcet (= cseg_off[n_tasks])                         */
+  int64_t n_gsegs;          /* length of gseg_misc and gseg_exec (= gseg_off[n_tasks])           */
+  const int64_t *task_off;  /* [n_tasksets+1]                                                    */
+  const int64_t *period;    /* [n_tasks]   T_i                                                   */
+  const int64_t *deadline;  /* [n_tasks]   D_i                                                   */
+  const int64_t *priority;  /* [n_tasks]   pi_i, larger = higher                                 */
+  const int64_t *core;      /* [n_tasks]   CPU core the task is partitioned to                   */
+  const int64_t *cseg_off;  /* [n_tasks+1]                                                       */
+  const int64_t *cseg_wcet; /* [n_csegs]   C_{i,k}                                               */
+  const int64_t *gseg_off;  /* [n_tasks+1]                                                       */
+  const int64_t *gseg_misc; /* [n_gsegs]   G^m_{i,j}                                             */
+  const int64_t *gseg_exec; /* [n_gsegs]   G^e_{i,j}                                             */
+} gcaps_tasksets_t;
+
+/*
+ * gcaps_rta_batch -- response-time analysis of a device-resident batch (Sec. 6: Eq. 1-4 and
+ * Lemmas 1-15; the fixed-point iteration is implied by R_i appearing on both sides of Eq. 1).
+ *
+ *   ts                      host struct whose pointers are DEVICE pointers (see above)
+ *   n_tasksets              number of tasksets, >= 0 (0 is a no-op)
+ *   policy                  GCAPS_POLICY_* | flags
+ *   timeslice_us            L of Eq. 3; used by RR only, must be 1..MAX_TIME there
+ *   ctx_switch_overhead_us  theta (Def. 1) for RR, epsilon = alpha + theta (Def. 2) for GCAPS;
+ *                           0..MAX_TIME
+ *   out_wcrt                DEVICE, [ts->n_tasks]: converged R_i, or a GCAPS_WCRT_* sentinel;
+ *                           indexed like the per-task input arrays
+ *   out_sched               DEVICE, [n_tasksets]: GCAPS_SCHED_*
+ *   workspace               DEVICE scratch of at least gcaps_rta_workspace_bytes() bytes, 256-byte
+ *                           aligned, caller-owned; contents are undefined afterwards.  It holds
+ *                           the size-binned launch plan (a permutation of taskset indices).
+ *   stream                  a cudaStream_t passed as void* (NULL = the default stream)
+ *
+ * For task i of a taskset, in decreasing priority:  R <- base_i;  repeat  R' <- base_i +
+ * sum over interfering (J, W, T_h) of ceil((R + J) / T_h) * W  until R' = R (converged, R_i = R)
+ * or R > D_i (MISS).  After the first MISS or ITER_LIMIT the remaining tasks are SKIPPED.
+ *
+ * Asynchronous: the work is enqueued on `stream`; no host synchronisation, no allocation.
+ * Returns GCAPS_OK or a negative GCAPS_ERR_* (nothing is enqueued on an argument error).
+ * Tasksets outside the input domain get GCAPS_SCHED_INVALID; the kernels never trap on them.
+ */
+int gcaps_rta_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
+                    int64_t timeslice_us, int64_t ctx_switch_overhead_us, int64_t *out_wcrt,
+                    uint8_t *out_sched, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * gcaps_rta_workspace_bytes -- size of the scratch buffer gcaps_rta_batch needs for a batch of
+ * n_tasksets tasksets (a pure host computation; 0 for a negative count).
+ */
+size_t gcaps_rta_workspace_bytes(int64_t n_tasksets);
+
+/*
+ * gcaps_rta_batch_host -- the same analysis for a batch held in HOST memory (task model: Sec. 4;
+ * analysis: Sec. 6).  `ts` holds host pointers, out_wcrt / out_sched are host arrays.  The call
+ * copies the inputs to the device in chunks of whole tasksets, runs gcaps_rta_batch on each
+ * chunk, copies the results back and returns after everything has completed.  Device staging
+ * memory is allocated on first use, grown on demand and kept until gcaps_rta_release_host();
+ * page-locked host buffers give the best transfer rate but are not required.
+ */
+int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
+                         int64_t timeslice_us, int64_t ctx_switch_overhead_us, int64_t *out_wcrt,
+                         uint8_t *out_sched);
+
+/* Frees the staging memory gcaps_rta_batch_host keeps on the current device. */
+void gcaps_rta_release_host(void);
+
+/*
+ * gcaps_rta_validate -- per-taskset check of the input domain stated above (task model: Sec. 4,
+ * D_i <= T_i).  out_err is a DEVICE array [n_tasksets]; 0 = valid, otherwise a bit mask of
+ * GCAPS_BAD_*.  Asynchronous on `stream`.
+ */
+#define GCAPS_BAD_TASK_RANGE 0x01 /* task_off not monotone / outside [0,n_tasks] / n too large  */
+#define GCAPS_BAD_SEG_RANGE 0x02  /* segment offsets not monotone / outside range / too many    */
+#define GCAPS_BAD_PERIOD 0x04     /* T_i outside 1..MAX_TIME                                     */
+#define GCAPS_BAD_DEADLINE 0x08   /* D_i outside 1..T_i                                          */
+#define GCAPS_BAD_CORE 0x10       /* core outside 0..MAX_CORE                                    */
+#define GCAPS_BAD_WCET 0x20       /* a segment WCET outside 0..MAX_TIME                          */
+int gcaps_rta_validate(const gcaps_tasksets_t *ts, int64_t n_tasksets, int32_t *out_err,
+                       void *stream);
+
+/* Text for a return code; never NULL. */
+const char *gcaps_rta_strerror(int code);
+
+/* The cudaError_t (as int) of the last failed CUDA call made by this library on this thread. */
+int gcaps_rta_last_cuda_error(void);
+
+/* GCAPS_RTA_VERSION of the loaded library. */
+int gcaps_rta_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GCAPS_RTA_H_ */

@@ -1,0 +1,53 @@
+"""ctypes wrapper of ``des_sim.c`` -- TEST INFRASTRUCTURE ONLY (see the package docstring)."""
+from __future__ import annotations
+
+import ctypes
+from typing import Sequence, Tuple
+
+import numpy as np
+
+from . import build as _build
+
+_p64 = ctypes.POINTER(ctypes.c_int64)
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build.build("des_sim"))
+        lib.des_simulate.argtypes = [ctypes.c_int] + [_p64] * 9 + [
+            ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_int64, _p64, _p64]
+        lib.des_simulate.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def simulate(batch, t: int, offsets: Sequence[int], policy: int, busy: bool, timeslice: int,
+             horizon: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Simulates taskset ``t`` of ``batch`` for ``horizon`` ticks.
+
+    Returns ``(max_resp, unfinished)`` per task: the largest response time of a completed job and
+    the age of a job still in progress at the horizon (0 if none).
+    """
+    lib = _load()
+    a, b = int(batch.task_off[t]), int(batch.task_off[t + 1])
+    n = b - a
+    c = lambda x: np.ascontiguousarray(x, dtype=np.int64)
+    T, prio, core = c(batch.period[a:b]), c(batch.priority[a:b]), c(batch.core[a:b])
+    off = c(offsets)
+    assert off.shape[0] == n
+    c_off = c(batch.cseg_off[a:b + 1] - batch.cseg_off[a])
+    g_off = c(batch.gseg_off[a:b + 1] - batch.gseg_off[a])
+    cs = c(batch.cseg_wcet[batch.cseg_off[a]:batch.cseg_off[b]])
+    gm = c(batch.gseg_misc[batch.gseg_off[a]:batch.gseg_off[b]])
+    ge = c(batch.gseg_exec[batch.gseg_off[a]:batch.gseg_off[b]])
+    max_resp = np.zeros(n, np.int64)
+    unfinished = np.zeros(n, np.int64)
+    p = lambda x: x.ctypes.data_as(_p64)
+    rc = lib.des_simulate(n, p(T), p(prio), p(core), p(off), p(c_off), p(cs), p(g_off), p(gm),
+                          p(ge), policy, 1 if busy else 0, timeslice, horizon, p(max_resp),
+                          p(unfinished))
+    if rc != 0:
+        raise ValueError("taskset does not fit the simulator's limits")
+    return max_resp, unfinished
