@@ -1,0 +1,184 @@
+"""Thin ctypes binding of the C-ABI library ``libgcaps_rta.so`` (declared in include/gcaps_rta.h).
+
+Argument marshalling only: every step of the analysis runs in the CUDA kernels of the library.
+PyTorch is used for device memory and streams.  There is no CPU fallback: if the library is
+missing or no B200 is present the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional, Tuple
+
+import numpy as np
+
+from . import build as _build
+from .taskgen import ARRAY_FIELDS, TasksetBatch
+
+POLICY_GCAPS = 0
+POLICY_RR = 1
+BUSY = 0x100
+LITERAL = 0x200
+
+SCHED_NO, SCHED_YES, SCHED_INVALID = 0, 1, 2
+WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID = -1, -2, -3, -4
+MAX_TASKS = 256
+MAX_TIME = 1 << 40
+
+OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NO_DEVICE = 0, -1, -2, -3, -4
+
+EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host",
+           "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
+           "gcaps_rta_last_cuda_error", "gcaps_rta_version")
+
+_p64 = ctypes.POINTER(ctypes.c_int64)
+
+
+class CTasksets(ctypes.Structure):
+    """Mirror of ``gcaps_tasksets_t``."""
+    _fields_ = [("n_tasks", ctypes.c_int64), ("n_csegs", ctypes.c_int64),
+                ("n_gsegs", ctypes.c_int64)] + [(f, ctypes.c_void_p) for f in ARRAY_FIELDS]
+
+
+class GcapsError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__("gcaps_rta: %s (code %d)" % (text, code))
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None):
+    """Loads libgcaps_rta.so (never builds it implicitly on a machine without the source
+    being newer: a missing library is an error, not a reason to fall back)."""
+    global _lib
+    if _lib is None or path is not None:
+        path = path or _build.CUDA_LIB
+        if not os.path.exists(path):
+            raise FileNotFoundError(
+                "%s is missing: run `python -m paper_2406_05221_b200.build` (needs nvcc)" % path)
+        lib = ctypes.CDLL(path)
+        lib.gcaps_rta_batch.argtypes = [
+            ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        lib.gcaps_rta_batch.restype = ctypes.c_int
+        lib.gcaps_rta_workspace_bytes.argtypes = [ctypes.c_int64]
+        lib.gcaps_rta_workspace_bytes.restype = ctypes.c_size_t
+        lib.gcaps_rta_batch_host.argtypes = [
+            ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_void_p]
+        lib.gcaps_rta_batch_host.restype = ctypes.c_int
+        lib.gcaps_rta_release_host.argtypes = []
+        lib.gcaps_rta_release_host.restype = None
+        lib.gcaps_rta_validate.argtypes = [ctypes.POINTER(CTasksets), ctypes.c_int64,
+                                           ctypes.c_void_p, ctypes.c_void_p]
+        lib.gcaps_rta_validate.restype = ctypes.c_int
+        lib.gcaps_rta_strerror.argtypes = [ctypes.c_int]
+        lib.gcaps_rta_strerror.restype = ctypes.c_char_p
+        lib.gcaps_rta_last_cuda_error.restype = ctypes.c_int
+        lib.gcaps_rta_version.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _check(rc: int):
+    if rc != OK:
+        lib = load_library()
+        text = lib.gcaps_rta_strerror(rc).decode()
+        if rc == ERR_CUDA:
+            text += " [cudaError %d]" % lib.gcaps_rta_last_cuda_error()
+        raise GcapsError(rc, text)
+
+
+def workspace_bytes(n_tasksets: int) -> int:
+    return int(load_library().gcaps_rta_workspace_bytes(n_tasksets))
+
+
+class DeviceTasksets:
+    """The ten input arrays as int64 CUDA tensors plus the C struct that points at them."""
+
+    def __init__(self, tensors: Dict[str, "torch.Tensor"]):
+        self.t = tensors
+        self.n_tasksets = int(tensors["task_off"].shape[0]) - 1
+        self.n_tasks = int(tensors["period"].shape[0])
+        self.n_csegs = int(tensors["cseg_wcet"].shape[0])
+        self.n_gsegs = int(tensors["gseg_misc"].shape[0])
+        self.c = CTasksets(self.n_tasks, self.n_csegs, self.n_gsegs,
+                           *[tensors[f].data_ptr() for f in ARRAY_FIELDS])
+
+    @staticmethod
+    def from_host(batch: TasksetBatch, device="cuda:0") -> "DeviceTasksets":
+        import torch
+        return DeviceTasksets({f: torch.from_numpy(np.ascontiguousarray(getattr(batch, f))).to(device)
+                               for f in ARRAY_FIELDS})
+
+    def input_bytes(self) -> int:
+        return sum(int(v.numel()) * 8 for v in self.t.values())
+
+
+def rta_batch(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, overhead_us: int = 0,
+              out_wcrt=None, out_sched=None, workspace=None, stream=None):
+    """gcaps_rta_batch on device-resident inputs.  Returns ``(out_wcrt, out_sched)`` CUDA tensors
+    (int64 per task, uint8 per taskset); asynchronous on ``stream`` (default: torch's current)."""
+    import torch
+    lib = load_library()
+    dev = ts.t["task_off"].device
+    with torch.cuda.device(dev):
+        if out_wcrt is None:
+            out_wcrt = torch.empty(ts.n_tasks, dtype=torch.int64, device=dev)
+        if out_sched is None:
+            out_sched = torch.empty(max(ts.n_tasksets, 0), dtype=torch.uint8, device=dev)
+        need = workspace_bytes(ts.n_tasksets)
+        if workspace is None:
+            workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        rc = lib.gcaps_rta_batch(ctypes.byref(ts.c), ts.n_tasksets, policy, timeslice_us, overhead_us,
+                                 out_wcrt.data_ptr(), out_sched.data_ptr(), workspace.data_ptr(),
+                                 workspace.numel(), st.cuda_stream)
+    _check(rc)
+    return out_wcrt, out_sched
+
+
+def rta_validate(ts: DeviceTasksets, stream=None):
+    """gcaps_rta_validate: int32 error mask per taskset (CUDA tensor)."""
+    import torch
+    lib = load_library()
+    dev = ts.t["task_off"].device
+    with torch.cuda.device(dev):
+        out = torch.empty(max(ts.n_tasksets, 0), dtype=torch.int32, device=dev)
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        rc = lib.gcaps_rta_validate(ctypes.byref(ts.c), ts.n_tasksets, out.data_ptr(), st.cuda_stream)
+    _check(rc)
+    return out
+
+
+def host_struct(arrays: Dict[str, np.ndarray]) -> Tuple[CTasksets, int]:
+    """C struct over host arrays (numpy int64, contiguous); returns (struct, n_tasksets)."""
+    for f in ARRAY_FIELDS:
+        a = arrays[f]
+        assert a.dtype == np.int64 and a.flags["C_CONTIGUOUS"], f
+    c = CTasksets(arrays["period"].shape[0], arrays["cseg_wcet"].shape[0],
+                  arrays["gseg_misc"].shape[0], *[arrays[f].ctypes.data for f in ARRAY_FIELDS])
+    return c, int(arrays["task_off"].shape[0]) - 1
+
+
+def rta_batch_host(arrays: Dict[str, np.ndarray], policy: int, timeslice_us: int = 1024,
+                   overhead_us: int = 0, out_wcrt: Optional[np.ndarray] = None,
+                   out_sched: Optional[np.ndarray] = None):
+    """gcaps_rta_batch_host on host arrays (page-locked ones transfer fastest).  Synchronous.
+    Returns ``(out_wcrt, out_sched)`` numpy arrays."""
+    lib = load_library()
+    c, n_tasksets = host_struct(arrays)
+    if out_wcrt is None:
+        out_wcrt = np.full(c.n_tasks, WCRT_INVALID, np.int64)
+    if out_sched is None:
+        out_sched = np.full(max(n_tasksets, 0), SCHED_INVALID, np.uint8)
+    rc = lib.gcaps_rta_batch_host(ctypes.byref(c), n_tasksets, policy, timeslice_us, overhead_us,
+                                  out_wcrt.ctypes.data, out_sched.ctypes.data)
+    _check(rc)
+    return out_wcrt, out_sched
+
+
+def release_host():
+    load_library().gcaps_rta_release_host()

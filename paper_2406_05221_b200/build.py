@@ -1,0 +1,49 @@
+"""In-tree build of the native sources: the CUDA library (nvcc, sm_100a) and the generator."""
+from __future__ import annotations
+
+import os
+import subprocess
+import sys
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+CUDA_SRC = os.path.join(_HERE, "csrc", "gcaps_rta.cu")
+CUDA_LIB = os.path.join(_HERE, "libgcaps_rta.so")
+HEADER = os.path.join(os.path.dirname(_HERE), "include", "gcaps_rta.h")
+
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+              "-shared", "-Xcompiler", "-fPIC"]
+
+
+def _nvcc() -> str:
+    for cand in (os.environ.get("NVCC"), "/usr/local/cuda/bin/nvcc", "nvcc"):
+        if cand and (os.path.isabs(cand) and os.path.exists(cand) or not os.path.isabs(cand)):
+            return cand
+    return "nvcc"
+
+
+def cuda_lib_is_stale() -> bool:
+    if not os.path.exists(CUDA_LIB):
+        return True
+    m = os.path.getmtime(CUDA_LIB)
+    return m < os.path.getmtime(CUDA_SRC) or m < os.path.getmtime(HEADER)
+
+
+def build_cuda(force: bool = False, verbose: bool = False) -> str:
+    """Compiles csrc/gcaps_rta.cu for sm_100a into libgcaps_rta.so beside this file."""
+    if force or cuda_lib_is_stale():
+        tmp = CUDA_LIB + ".%d.tmp" % os.getpid()
+        cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp, CUDA_SRC]
+        subprocess.check_call(cmd)
+        os.replace(tmp, CUDA_LIB)
+    return CUDA_LIB
+
+
+def build_all(force: bool = False) -> None:
+    from . import taskgen
+    taskgen.build_taskgen(force)
+    build_cuda(force)
+
+
+if __name__ == "__main__":
+    build_all(force="--force" in sys.argv)
+    print(CUDA_LIB)

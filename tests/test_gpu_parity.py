@@ -1,0 +1,255 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, through the C-ABI.
+
+All times are integer microseconds, so the bar is bit-exact equality of every out_wcrt value
+(including the sentinels) and every out_sched flag.
+"""
+import copy
+import ctypes
+
+import numpy as np
+import pytest
+
+from oracle import rta
+from paper_2406_05221_b200 import binding, taskgen
+from tests.helpers import ALL_MODES, BUSY, LITERAL, batch_of, parse_vectors, random_tasksets
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+MODES4 = [0, BUSY, 1, 1 | BUSY]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    binding.load_library()
+
+
+def gpu_run(batch, policy, L=1024, ovh=0):
+    ts = binding.DeviceTasksets.from_host(batch)
+    wcrt = torch.full((ts.n_tasks,), binding.WCRT_INVALID, dtype=torch.int64, device="cuda")
+    sched = torch.full((max(ts.n_tasksets, 0),), binding.SCHED_INVALID, dtype=torch.uint8, device="cuda")
+    binding.rta_batch(ts, policy, L, ovh, out_wcrt=wcrt, out_sched=sched)
+    torch.cuda.synchronize()
+    return wcrt.cpu().numpy(), sched.cpu().numpy()
+
+
+def assert_parity(batch, policy, L=1024, ovh=0, what=""):
+    w_ref, s_ref, _ = rta.analyse(batch, policy, L, ovh)
+    w, s = gpu_run(batch, policy, L, ovh)
+    bad_s = np.nonzero(s != s_ref)[0]
+    assert bad_s.size == 0, "%s: out_sched differs at tasksets %s" % (what, bad_s[:5])
+    bad_w = np.nonzero(w != w_ref)[0]
+    assert bad_w.size == 0, "%s: out_wcrt differs at tasks %s: %s vs oracle %s" % (
+        what, bad_w[:5], w[bad_w[:5]], w_ref[bad_w[:5]])
+    return w, s
+
+
+@pytest.mark.parametrize("fixture", ["table2_vectors.txt", "indirect_delay_vectors.txt"])
+def test_hand_derived_vectors(fixture):
+    tasks, cases = parse_vectors(fixture)
+    b = batch_of([tasks])
+    for c in cases:
+        w, s = gpu_run(b, c["policy"], c["L"], c["ovh"])
+        assert w.tolist() == c["expect"], c["name"]
+
+
+@pytest.mark.parametrize("policy", ALL_MODES)
+def test_random_small_tasksets_all_modes(policy):
+    rng = np.random.default_rng(policy + 11)
+    sets = random_tasksets(rng, 3000, max_tasks=12, max_cores=4, wcet_hi=8)
+    sets += random_tasksets(rng, 500, max_tasks=12, unique_prio=False)
+    b = batch_of(sets)
+    for L, ovh in ((1, 0), (3, 1), (7, 2)):
+        assert_parity(b, policy, L, ovh, "random small")
+
+
+@pytest.mark.parametrize("name,count", [("pr1", 1000), ("sweep", 3000), ("large", 1500),
+                                        ("rr_model", 3000), ("divergence", 6000)])
+def test_workload_samples(name, count):
+    """The five benchmark workloads, several tiles and a ragged tail each."""
+    w = taskgen.WORKLOADS[name]
+    for stream in sorted({0, len(w.streams) // 2, len(w.streams) - 1}):
+        b = w.generate(7, count - 3, stream=stream)
+        modes = MODES4 if "gcaps" in w.policies else [1, 1 | BUSY]
+        for policy in modes:
+            wc, s = assert_parity(b, policy, w.timeslice_us, w.overhead_us, "%s/%d" % (name, stream))
+        if name in ("pr1", "sweep") and stream == 0:
+            assert s.max() == 1  # the easy end of the sweep has schedulable tasksets
+
+
+def test_rr_driver_model_grid():
+    w = taskgen.WORKLOADS["rr_model"]
+    b = w.generate(0, 1500)
+    for L in w.timeslices:
+        for theta in w.overheads:
+            assert_parity(b, 1, L, theta, "rr grid L=%d theta=%d" % (L, theta))
+
+
+def test_zero_overhead_and_literal_on_workloads():
+    b = taskgen.WORKLOADS["sweep"].generate(0, 1500, stream=2)
+    for policy in ALL_MODES:
+        assert_parity(b, policy, 1024, 0, "sweep ovh=0")
+        assert_parity(b, policy, 1000, 200, "sweep ovh=200")
+
+
+def test_size_bins_and_edges():
+    """Sizes around every bin boundary, empty tasksets, the maximum size, in one batch."""
+    rng = np.random.default_rng(5)
+    sets = []
+    for n in (0, 1, 2, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 95, 96, 97, 128, 200, 255, 256, 0, 3):
+        ts = []
+        for i in range(n):
+            T = int(rng.integers(2000, 200000))
+            ng = int(rng.integers(0, 3))
+            ts.append(dict(T=T, D=T - int(rng.integers(0, T // 4)), prio=int(rng.integers(0, 50)),
+                           core=int(rng.integers(0, 9)),
+                           cseg=[int(rng.integers(0, max(2, T // (40 * max(n, 1))))) for _ in range(ng + 1)],
+                           gseg=[(int(rng.integers(0, 5)), int(rng.integers(0, max(2, T // (60 * max(n, 1))))))
+                                 for _ in range(ng)]))
+        sets.append(ts)
+    b = batch_of(sets)
+    for policy in ALL_MODES:
+        assert_parity(b, policy, 64, 3, "bins")
+    # reversed order exercises another permutation of the plan
+    b2 = batch_of(sets[::-1])
+    assert_parity(b2, 0, 64, 3, "bins reversed")
+
+
+def test_empty_batch_and_empty_arrays():
+    b = batch_of([])
+    w, s = gpu_run(b, 0)
+    assert w.size == 0 and s.size == 0
+    b = batch_of([[], [], []])
+    w, s = gpu_run(b, 1, 5, 1)
+    assert s.tolist() == [1, 1, 1]
+
+
+def test_invalid_tasksets_are_flagged_not_trapped():
+    good = [dict(T=10, prio=1, core=0, cseg=[1], gseg=[(1, 2)])]
+    sets = [good,
+            [dict(T=10, D=11, prio=1, core=0, cseg=[1]), dict(T=10, prio=0, core=0, cseg=[1])],
+            [dict(T=10, prio=1, core=0, cseg=[-1])],
+            [],
+            [dict(T=10, prio=1, core=-1, cseg=[1])],
+            [dict(T=0, D=0, prio=1, core=0, cseg=[1])],
+            [dict(T=(1 << 40) + 1, prio=1, core=0, cseg=[1])],
+            [dict(T=100, prio=1, core=0, cseg=[1], gseg=[(0, (1 << 40) + 1)])],
+            [dict(T=100, prio=i, core=0, cseg=[1]) for i in range(257)],
+            good]
+    b = batch_of(sets)
+    for policy in (0, 1 | BUSY):
+        w, s = assert_parity(b, policy, 4, 0, "invalid")
+    assert s.tolist() == [1, 2, 2, 1, 2, 2, 2, 2, 2, 1]
+    err = binding.rta_validate(binding.DeviceTasksets.from_host(b)).cpu().numpy()
+    assert err.tolist() == rta.validate(b).tolist()
+    # broken offsets: the oracle and the library agree and nothing faults
+    for field, idx, val in (("task_off", 2, 9999), ("task_off", 3, -4), ("cseg_off", 2, -1),
+                            ("gseg_off", 1, 1 << 50), ("cseg_off", 5, 0)):
+        bb = copy.deepcopy(b)
+        getattr(bb, field)[idx] = val
+        w_ref, s_ref, _ = rta.analyse(bb, 0, 4, 0)
+        w, s = gpu_run(bb, 0, 4, 0)
+        assert (s == s_ref).all(), (field, idx)
+        assert (w == w_ref).all(), (field, idx)
+        err = binding.rta_validate(binding.DeviceTasksets.from_host(bb)).cpu().numpy()
+        assert err.tolist() == rta.validate(bb).tolist()
+
+
+def test_iteration_cap_and_extreme_values():
+    B = 1 << 40
+    sets = [
+        [dict(T=2, prio=2, core=0, cseg=[2]), dict(T=1 << 23, prio=1, core=0, cseg=[1])],  # ITER_LIMIT
+        [dict(T=2, prio=2, core=0, cseg=[2]), dict(T=1001, prio=1, core=0, cseg=[1])],     # slow miss
+        [dict(T=B, prio=3, core=0, cseg=[B // 8], gseg=[(B // 16, B // 16)]),
+         dict(T=B, prio=2, core=0, cseg=[B // 16], gseg=[(1, B // 16)]),
+         dict(T=B, prio=1, core=1, cseg=[B // 2], gseg=[(0, 1)])],
+        [dict(T=B, prio=1, core=0, cseg=[B >> 10] * 512, gseg=[(B >> 12, B >> 12)] * 512)],
+        [dict(T=1, prio=2, core=0, cseg=[1]), dict(T=5, prio=1, core=0, cseg=[1])],
+        [dict(T=50, prio=2, core=0, cseg=[0]), dict(T=50, prio=1, core=0, cseg=[0], gseg=[(0, 0)])],
+    ]
+    b = batch_of(sets)
+    for policy in ALL_MODES:
+        w, s = assert_parity(b, policy, 1, 0, "extreme")
+        assert_parity(b, policy, 1, B, "extreme ovh")
+        assert_parity(b, policy, B, 1, "extreme L")
+    w, s = gpu_run(b, 0, 1, 0)
+    assert w[1] == binding.WCRT_ITER_LIMIT and w[3] == binding.WCRT_MISS
+
+
+def test_determinism_and_output_reuse():
+    b = taskgen.WORKLOADS["divergence"].generate(1000, 4000)
+    ts = binding.DeviceTasksets.from_host(b)
+    outs = []
+    for _ in range(3):
+        w, s = binding.rta_batch(ts, 0, 1024, 50)
+        torch.cuda.synchronize()
+        outs.append((w.cpu().numpy().copy(), s.cpu().numpy().copy()))
+    for w, s in outs[1:]:
+        assert (w == outs[0][0]).all() and (s == outs[0][1]).all()
+
+
+def test_streams_and_workspace_errors():
+    b = taskgen.WORKLOADS["pr1"].generate(0, 300)
+    ts = binding.DeviceTasksets.from_host(b)
+    w_ref, s_ref, _ = rta.analyse(b, 0, 1024, 50)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        w, s = binding.rta_batch(ts, 0, 1024, 50)
+    side.synchronize()
+    assert (w.cpu().numpy() == w_ref).all() and (s.cpu().numpy() == s_ref).all()
+    tiny = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.GcapsError) as e:
+        binding.rta_batch(ts, 0, 1024, 50, workspace=tiny)
+    assert e.value.code == binding.ERR_WORKSPACE
+    with pytest.raises(binding.GcapsError):
+        binding.rta_batch(ts, 1, 0, 0)
+
+
+def test_host_buffer_entry_point():
+    """gcaps_rta_batch_host: chunked copies in, analysis, copies out -- same results."""
+    b = taskgen.WORKLOADS["divergence"].generate(0, 150_000)   # several chunks
+    for policy in (0, 1):
+        w_ref, s_ref, _ = rta.analyse(b, policy, 1024, 50)
+        w, s = binding.rta_batch_host(b.arrays(), policy, 1024, 50)
+        assert (s == s_ref).all() and (w == w_ref).all()
+    # pinned buffers, and a batch with malformed offsets in the middle
+    small = taskgen.WORKLOADS["sweep"].generate(0, 500)
+    pinned = {f: torch.from_numpy(a.copy()).pin_memory().numpy() for f, a in small.arrays().items()}
+    w_ref, s_ref, _ = rta.analyse(small, 1 | BUSY, 512, 25)
+    w, s = binding.rta_batch_host(pinned, 1 | BUSY, 512, 25)
+    assert (s == s_ref).all() and (w == w_ref).all()
+    broken = copy.deepcopy(small)
+    broken.cseg_off[broken.task_off[200] + 3] = -7
+    broken.task_off[400] = broken.task_off[399] - 1
+    w_ref, s_ref, _ = rta.analyse(broken, 0, 512, 25)
+    w, s = binding.rta_batch_host(broken.arrays(), 0, 512, 25)
+    assert (s == s_ref).all() and (w == w_ref).all()
+    binding.release_host()
+
+
+def test_full_size_large_workload_sampled():
+    """The benchmark's own configuration (1,000,000 tasksets of 80 tasks): outputs of sampled
+    tasksets against the oracle, and properties that hold at any size for the rest."""
+    w = taskgen.WORKLOADS["large"]
+    b = w.generate(0, w.n_tasksets)
+    ts = binding.DeviceTasksets.from_host(b)
+    rng = np.random.default_rng(9)
+    sample = np.sort(rng.choice(w.n_tasksets, 3000, replace=False))
+    sub = b.select(sample)
+    for policy in (0, 1):
+        wc, sc = binding.rta_batch(ts, policy, w.timeslice_us, w.overhead_us)
+        torch.cuda.synchronize()
+        wc, sc = wc.cpu().numpy().reshape(-1, 80), sc.cpu().numpy()
+        w_ref, s_ref, _ = rta.analyse(sub, policy, w.timeslice_us, w.overhead_us)
+        assert (sc[sample] == s_ref).all()
+        assert (wc[sample].reshape(-1) == w_ref).all()
+        # any size: flags are 0/1; schedulable <=> no sentinel; at most one MISS per taskset
+        assert sc.max() <= 1
+        has_neg = (wc < 0).any(axis=1)
+        assert ((sc == 1) == ~has_neg).all()
+        assert ((wc == binding.WCRT_MISS).sum(axis=1) <= 1).all()
+        D = b.deadline.reshape(-1, 80)
+        ok = wc >= 0
+        assert (wc[ok] <= D[ok]).all()
