@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Throughput benchmark of the batched response-time analysis (tasksets analysed per second).
+
+A step is one pass of the whole hot path over one batch of synthetic tasksets: the GCAPS
+analysis and the round-robin analysis of every taskset of the batch (two library calls).  The
+default workload is the 1,000,000-taskset configuration (8 cores x 10 tasks per taskset).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run, one rank per GPU)
+every rank analyses its own shard of the generator stream; there is no data-path collective.
+`--impl reference` times the CPU oracle on a bounded sample instead (host cores, no GPU).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tasksets analysed/sec (GCAPS & RR RTA)"
+UNIT = "tasksets/s"
+FALLBACK_HBM_GBS = 6650.0
+# plain-ALU peak of one B200: 148 SMs x 128 INT32 lanes x 1.965 GHz (integer lane-operations/s)
+ALU_PEAK_LANEOPS = 148 * 128 * 1.965e9
+K_TERM, K_SETUP = 6, 16   # algorithmic integer lane-operations per interference term / per task
+# kernels launched by one gcaps_rta_batch call: 3 plan kernels + one analysis kernel per size bin
+LAUNCHES_PER_CALL = 9
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id, self.proc = gpu_id, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.gpu_id, "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in text.strip().splitlines():
+            tok = [x.strip() for x in line.split(",")]
+            if len(tok) < 7:
+                continue
+            try:
+                sm.append(float(tok[0]))
+                mx.append(float(tok[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, tok[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def oracle_sample(workload, first, count, budget_s, chunk=50_000):
+    """Times the CPU oracle (as it stands, one thread) on tasksets first.. of the workload, both
+    policies per taskset, stopping after ``count`` tasksets or ``budget_s`` seconds."""
+    from oracle import rta
+    done, spent, terms, sweeps, started = 0, 0.0, [0, 0], [0, 0], [0, 0]
+    while done < count and spent < budget_s:
+        n = min(chunk, count - done)
+        batch = workload.generate(first + done, n)
+        t0 = time.perf_counter()
+        for k, policy in enumerate((rta.POLICY_GCAPS, rta.POLICY_RR)):
+            _, _, c = rta.analyse(batch, policy, workload.timeslice_us, workload.overhead_us)
+            terms[k] += c.terms
+            sweeps[k] += c.sweeps
+            started[k] += c.tasks
+        spent += time.perf_counter() - t0
+        done += n
+    return {"tasksets": done, "seconds": spent, "terms": terms, "sweeps": sweeps, "started": started}
+
+
+def run_reference(args, workload):
+    """The reference arm: the CPU oracle, single-threaded, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = min(args.ref_sample, workload.n_tasksets)
+    for _ in range(args.warmup):
+        oracle_sample(workload, 0, min(per_step, 10_000), 1e9)
+    t_total, n_total = 0.0, 0
+    for k in range(args.steps):
+        r = oracle_sample(workload, (k * per_step) % max(1, workload.n_tasksets - per_step + 1), per_step, 1e9)
+        t_total += r["seconds"]
+        n_total += r["tasksets"]
+    value = n_total / t_total
+    sample = "%d tasksets of '%s' per step, both policies, generation excluded" % (per_step, workload.name)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+        "data": "synthetic", "config": {"workload": workload.name, "tasksets_per_step": per_step,
+                                         "note": workload.note},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large")
+    ap.add_argument("--stream", type=int, default=0, help="sweep point of the workload")
+    ap.add_argument("--tasksets", type=int, default=0, help="tasksets per GPU (0 = the workload's own size)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--ref-sample", type=int, default=100_000)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2406_05221_b200 import taskgen
+    workload = taskgen.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, workload)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2406_05221_b200 import binding, sharding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    binding.load_library()
+
+    per_gpu = args.tasksets or workload.n_tasksets
+    first, count = sharding.weak_shard(rank, per_gpu)
+    pinned = []
+
+    def alloc(n):
+        t = torch.empty(max(n, 1), dtype=torch.int64, pin_memory=True)
+        pinned.append(t)
+        return t.numpy()[:n]
+
+    batch = workload.generate(first, count, stream=args.stream, alloc=alloc)
+    ts = binding.DeviceTasksets.from_host(batch, dev)
+    out_wcrt = torch.empty(ts.n_tasks, dtype=torch.int64, device=dev)
+    out_sched = torch.empty(ts.n_tasksets, dtype=torch.uint8, device=dev)
+    workspace = torch.empty(max(256, binding.workspace_bytes(ts.n_tasksets)), dtype=torch.uint8, device=dev)
+    policies = [p for p in (binding.POLICY_GCAPS, binding.POLICY_RR)
+                if ("gcaps", "rr")[p] in workload.policies]
+    names = [("gcaps", "rr")[p] for p in policies]
+    L, ovh = workload.timeslice_us, workload.overhead_us
+    stream = torch.cuda.current_stream(dev)
+
+    def step(events=None):
+        for k, policy in enumerate(policies):
+            if events is not None:
+                events[k].record(stream)
+            binding.rta_batch(ts, policy, L, ovh, out_wcrt=out_wcrt, out_sched=out_sched,
+                              workspace=workspace, stream=stream)
+        if events is not None:
+            events[len(policies)].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(policies) + 1)] for _ in range(args.steps)]
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    barrier()
+    sampler.start()
+    t_wall0 = time.perf_counter()
+    for k in range(args.steps):
+        step(ev[k])
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    total_ms = ev[0][0].elapsed_time(ev[-1][-1])
+    per_policy_ms = [statistics.mean(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(len(policies))]
+    best_policy_ms = [min(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(len(policies))]
+    sched_frac = float((out_sched == 1).float().mean().item()) if count else 0.0
+    total_ms = sharding.reduce_scalars([total_ms], "max", dev)[0]
+    ms_per_step = total_ms / args.steps
+    value = world * count / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (copies inside the timed region) -----
+    e2e = None
+    if not args.no_e2e:
+        host_wcrt = torch.empty(max(ts.n_tasks, 1), dtype=torch.int64, pin_memory=True).numpy()[:ts.n_tasks]
+        host_sched = torch.empty(max(ts.n_tasksets, 1), dtype=torch.uint8, pin_memory=True).numpy()[:ts.n_tasksets]
+        arrays = batch.arrays()
+        for policy in policies:  # warm-up: staging buffers get allocated here
+            binding.rta_batch_host(arrays, policy, L, ovh, host_wcrt, host_sched)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            for policy in policies:
+                binding.rta_batch_host(arrays, policy, L, ovh, host_wcrt, host_sched)
+        barrier()
+        dt = time.perf_counter() - t0
+        dt = sharding.reduce_scalars([dt], "max", dev)[0]
+        e2e = {"value": world * count * args.e2e_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": len(policies) * batch.input_bytes(),
+               "d2h_bytes_per_step": len(policies) * batch.output_bytes(),
+               "steps": args.e2e_steps, "ms_per_step": 1e3 * dt / args.e2e_steps,
+               "api": "gcaps_rta_batch_host, page-locked host arrays, one call per policy"}
+        binding.release_host()
+
+    # ---- the oracle beside it, and the roofline of the dominant launch ------------------------
+    cpu = None
+    bytes_per_call = batch.input_bytes() + batch.output_bytes()
+    peak, peak_kind = measured_peaks()
+    roof = None
+    if rank == 0:
+        dom = int(np.argmax(per_policy_ms))
+        achieved = bytes_per_call / (per_policy_ms[dom] * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
+                "kernel": "analysis kernel of the %s call (the call's plan kernels are inside the timing)"
+                          % names[dom].upper(),
+                "algorithmic_bytes_per_launch": bytes_per_call,
+                "ms_per_launch": dict(zip(names, per_policy_ms)),
+                "best_ms_per_launch": dict(zip(names, best_policy_ms)),
+                "frac_per_policy": {nm: bytes_per_call / (ms * 1e-3) / 1e9 / peak
+                                    for nm, ms in zip(names, per_policy_ms)}}
+        if world == 1 and not args.no_cpu_baseline:
+            r = oracle_sample(workload, first, count, args.cpu_budget)
+            cpu = {"value": r["tasksets"] / r["seconds"], "unit": UNIT, "cores": 1, "kind": "oracle",
+                   "sample": "first %d tasksets of the workload, both policies, %.1f s, generation excluded"
+                             % (r["tasksets"], r["seconds"]),
+                   "terms_per_taskset": {"gcaps": r["terms"][0] / r["tasksets"], "rr": r["terms"][1] / r["tasksets"]}}
+            # which roofline binds: algorithmic integer work against algorithmic bytes
+            n_tasks_per_set = ts.n_tasks / max(1, ts.n_tasksets)
+            t_mem = bytes_per_call / (peak * 1e9)
+            pol_idx = policies[dom]
+            t_alu = count * (K_TERM * r["terms"][pol_idx] / r["tasksets"] + K_SETUP * n_tasks_per_set) / ALU_PEAK_LANEOPS
+            roof["model_ms"] = {"hbm": 1e3 * t_mem, "alu": 1e3 * t_alu}
+            if t_alu > t_mem:
+                ops = t_alu * ALU_PEAK_LANEOPS
+                ach = ops / (per_policy_ms[dom] * 1e-3)
+                roof.update(bound="alu", achieved=ach / 1e12, peak=ALU_PEAK_LANEOPS / 1e12,
+                            unit="Tlaneop/s", frac=ach / ALU_PEAK_LANEOPS)
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": workload.name, "note": workload.note, "tasksets_per_gpu": count,
+                       "tasks": ts.n_tasks, "policies": names, "mode": "self-suspension",
+                       "timeslice_us": L, "overhead_us": ovh,
+                       "analyses_per_taskset_per_step": len(policies),
+                       "l2": "inputs (%.2f GB per call) against a 126 MB L2; no flush between steps"
+                             % (batch.input_bytes() / 1e9),
+                       "schedulable_fraction_last_policy": sched_frac,
+                       "input_checksum": batch.checksum() if count <= 200_000 else None},
+            "clocks": clocks, "e2e": e2e,
+            "gpu_launches": args.steps * len(policies) * LAUNCHES_PER_CALL,
+            "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -239,8 +239,11 @@ def _ranges(start: np.ndarray, length: np.ndarray) -> np.ndarray:
     return np.cumsum(out)
 
 
-def generate(params: GenParams, first: int, count: int, threads: Optional[int] = None) -> TasksetBatch:
-    """Tasksets ``first .. first+count-1`` of the stream described by ``params``."""
+def generate(params: GenParams, first: int, count: int, threads: Optional[int] = None,
+             alloc=None) -> TasksetBatch:
+    """Tasksets ``first .. first+count-1`` of the stream described by ``params``.
+
+    ``alloc(n)`` may supply the int64 output arrays (e.g. views of page-locked memory)."""
     lib = _load()
     if count <= 0:
         return TasksetBatch.from_tasksets([])
@@ -254,14 +257,12 @@ def generate(params: GenParams, first: int, count: int, threads: Optional[int] =
     starts = np.zeros((count, 3), np.int64)
     np.cumsum(counts[:-1], axis=0, out=starts[1:])
     n_tasks, n_c, n_g = (int(x) for x in counts.sum(axis=0))
-    arr = {
-        "task_off": np.empty(count + 1, np.int64),
-        "period": np.empty(n_tasks, np.int64), "deadline": np.empty(n_tasks, np.int64),
-        "priority": np.empty(n_tasks, np.int64), "core": np.empty(n_tasks, np.int64),
-        "cseg_off": np.empty(n_tasks + 1, np.int64), "cseg_wcet": np.empty(n_c, np.int64),
-        "gseg_off": np.empty(n_tasks + 1, np.int64), "gseg_misc": np.empty(n_g, np.int64),
-        "gseg_exec": np.empty(n_g, np.int64),
-    }
+    if alloc is None:
+        alloc = lambda n: np.empty(n, np.int64)
+    sizes = {"task_off": count + 1, "period": n_tasks, "deadline": n_tasks, "priority": n_tasks,
+             "core": n_tasks, "cseg_off": n_tasks + 1, "cseg_wcet": n_c, "gseg_off": n_tasks + 1,
+             "gseg_misc": n_g, "gseg_exec": n_g}
+    arr = {f: alloc(sizes[f]) for f in ARRAY_FIELDS}
     lib.tg_fill(ctypes.byref(cp), first, count, ptr(starts), *[ptr(arr[f]) for f in ARRAY_FIELDS])
     return TasksetBatch(**arr)
 
@@ -279,10 +280,11 @@ class Workload:
     policies: Sequence[str] = ("gcaps", "rr")
     note: str = ""
 
-    def generate(self, first: int = 0, count: Optional[int] = None, stream: int = 0) -> TasksetBatch:
+    def generate(self, first: int = 0, count: Optional[int] = None, stream: int = 0,
+                 alloc=None) -> TasksetBatch:
         if count is None:
             count = self.n_tasksets - first
-        return generate(self.streams[stream], first, count)
+        return generate(self.streams[stream], first, count, alloc=alloc)
 
 
 def _workloads() -> Dict[str, Workload]:
