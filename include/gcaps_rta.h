@@ -68,6 +68,8 @@ extern "C" {
 #define GCAPS_ERR_WORKSPACE (-2)     /* workspace null or smaller than gcaps_rta_workspace_bytes */
 #define GCAPS_ERR_CUDA (-3)          /* a CUDA runtime call failed; see gcaps_rta_last_cuda_error */
 #define GCAPS_ERR_NO_DEVICE (-4)     /* no CUDA device / not an sm_100 device                    */
+#define GCAPS_ERR_TOO_LARGE (-5)     /* batch larger than GCAPS_RTA_STATIC_MAX_TASKSETS (only
+                                        returned by gcaps_rta_batch_static)                     */
 
 /*
  * A batch of tasksets in CSR structure-of-arrays form (task model: Sec. 4).
@@ -153,6 +155,38 @@ size_t gcaps_rta_workspace_bytes(int64_t n_tasksets);
 int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
                          int64_t timeslice_us, int64_t ctx_switch_overhead_us, int64_t *out_wcrt,
                          uint8_t *out_sched);
+
+/*
+ * gcaps_rta_batch_static -- gcaps_rta_batch for callers that are not able to allocate device
+ * memory.  (The paper has no counterpart: this is a convenience of this library, not a step of
+ * the analysis.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plug-in inside a host
+ * application that owns the allocator and hands out only input and output buffers, a real-time
+ * or safety-certified process that must not allocate after start-up, or a caller in a context
+ * where an allocation would synchronise the device or fail outright.  Such a caller cannot
+ * provide the workspace gcaps_rta_batch asks for.  Here the workspace is a fixed array that is
+ * part of the library image itself: every GPU that loads the library holds
+ * GCAPS_RTA_STATIC_SCRATCH_BYTES of device memory for it until the process exits.
+ *
+ * Arguments, results, error codes and asynchrony are those of gcaps_rta_batch, minus the two
+ * workspace arguments, with these differences:
+ *   - n_tasksets may not exceed GCAPS_RTA_STATIC_MAX_TASKSETS; a larger batch is refused with
+ *     GCAPS_ERR_TOO_LARGE and nothing is enqueued (split the batch, or use gcaps_rta_batch);
+ *   - the call allocates nothing and frees nothing, on the host or on the device;
+ *   - the first call on each device looks up the device address of the array (one cheap runtime
+ *     query with that device current).  Make that first call outside any stream capture;
+ *   - every call on a device shares the one array and finds the previous call's plan in it.
+ *     The kernels rewrite every word of it that they later read, so stale contents are harmless,
+ *     but two calls whose kernels overlap on the GPU (different streams, or different host
+ *     threads without ordering) race on it and give undefined results.  Calls issued to one
+ *     stream, or otherwise ordered, are safe.
+ */
+#define GCAPS_RTA_STATIC_MAX_TASKSETS 65536
+#define GCAPS_RTA_STATIC_SCRATCH_BYTES (256 + 2048 + 4 * GCAPS_RTA_STATIC_MAX_TASKSETS)
+int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
+                           int64_t timeslice_us, int64_t ctx_switch_overhead_us,
+                           int64_t *out_wcrt, uint8_t *out_sched, void *stream);
 
 /* Frees the staging memory gcaps_rta_batch_host keeps on the current device. */
 void gcaps_rta_release_host(void);

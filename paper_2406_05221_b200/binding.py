@@ -25,11 +25,12 @@ WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID = -1, -2, -3, -4
 MAX_TASKS = 256
 MAX_TIME = 1 << 40
 
-OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NO_DEVICE = 0, -1, -2, -3, -4
+OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NO_DEVICE, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5
+STATIC_MAX_TASKSETS = 65536
 
 EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host",
            "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
-           "gcaps_rta_last_cuda_error", "gcaps_rta_version")
+           "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static")
 
 _p64 = ctypes.POINTER(ctypes.c_int64)
 
@@ -63,6 +64,10 @@ def load_library(path: Optional[str] = None):
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         lib.gcaps_rta_batch.restype = ctypes.c_int
+        lib.gcaps_rta_batch_static.argtypes = [
+            ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.gcaps_rta_batch_static.restype = ctypes.c_int
         lib.gcaps_rta_workspace_bytes.argtypes = [ctypes.c_int64]
         lib.gcaps_rta_workspace_bytes.restype = ctypes.c_size_t
         lib.gcaps_rta_batch_host.argtypes = [
@@ -136,6 +141,31 @@ def rta_batch(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, overhea
         rc = lib.gcaps_rta_batch(ctypes.byref(ts.c), ts.n_tasksets, policy, timeslice_us, overhead_us,
                                  out_wcrt.data_ptr(), out_sched.data_ptr(), workspace.data_ptr(),
                                  workspace.numel(), st.cuda_stream)
+    _check(rc)
+    return out_wcrt, out_sched
+
+
+def rta_batch_static(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, overhead_us: int = 0,
+                     out_wcrt=None, out_sched=None, stream=None):
+    """gcaps_rta_batch_static: the same analysis for callers that cannot allocate device memory.
+
+    The library's built-in scratch array takes the place of the workspace, so the call itself
+    allocates nothing; this wrapper only creates the two output tensors when the caller passes
+    none.  At most ``STATIC_MAX_TASKSETS`` tasksets per call (``GcapsError`` with
+    ``ERR_TOO_LARGE`` beyond).  Calls that could overlap on the GPU must be ordered by the caller:
+    they share the one scratch array."""
+    import torch
+    lib = load_library()
+    dev = ts.t["task_off"].device
+    with torch.cuda.device(dev):
+        if out_wcrt is None:
+            out_wcrt = torch.empty(ts.n_tasks, dtype=torch.int64, device=dev)
+        if out_sched is None:
+            out_sched = torch.empty(max(ts.n_tasksets, 0), dtype=torch.uint8, device=dev)
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        rc = lib.gcaps_rta_batch_static(ctypes.byref(ts.c), ts.n_tasksets, policy, timeslice_us,
+                                        overhead_us, out_wcrt.data_ptr(), out_sched.data_ptr(),
+                                        st.cuda_stream)
     _check(rc)
     return out_wcrt, out_sched
 

@@ -569,6 +569,12 @@ struct HostStage {
 };
 HostStage g_stage = {{nullptr, nullptr}, {0, 0}, {nullptr, nullptr}, -1, false};
 
+// Workspace of gcaps_rta_batch_static: lives in the library image, one copy per device that
+// loads it.  In host code this name is only a handle for cudaGetSymbolAddress, never an address
+// a kernel may be given.
+static __device__ __align__(256) unsigned char g_static_scratch[GCAPS_RTA_STATIC_SCRATCH_BYTES];
+void *g_static_scratch_ptr[64];  // device address of the array, per device, once looked up
+
 }  // namespace
 
 extern "C" {
@@ -593,6 +599,44 @@ int gcaps_rta_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
   KParams p;
   fill_params(&p, ts, n_tasksets, policy, timeslice_us, ctx_switch_overhead_us, out_wcrt, out_sched);
   return enqueue_batch(p, workspace, workspace_bytes, di.sm_count, (cudaStream_t)stream);
+}
+
+int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
+                           int64_t timeslice_us, int64_t ctx_switch_overhead_us,
+                           int64_t *out_wcrt, uint8_t *out_sched, void *stream) {
+  int rc = check_args(ts, n_tasksets, policy, timeslice_us, ctx_switch_overhead_us);
+  if (rc != GCAPS_OK) return rc;
+  if (n_tasksets > GCAPS_RTA_STATIC_MAX_TASKSETS ||
+      gcaps_rta_workspace_bytes(n_tasksets) > (size_t)GCAPS_RTA_STATIC_SCRATCH_BYTES)
+    return GCAPS_ERR_TOO_LARGE;
+  if (n_tasksets == 0) return GCAPS_OK;
+  if (!out_sched || (ts->n_tasks > 0 && !out_wcrt)) return GCAPS_ERR_INVALID_ARG;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != GCAPS_OK) return rc;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= 64) {
+    g_last_cuda_error = (int)e;
+    return GCAPS_ERR_NO_DEVICE;
+  }
+  if (!g_static_scratch_ptr[dev]) {
+    // once per device, with that device current: the array's address on this device
+    void *ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      g_last_cuda_error = (int)e;
+      return GCAPS_ERR_CUDA;
+    }
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  KParams p;
+  fill_params(&p, ts, n_tasksets, policy, timeslice_us, ctx_switch_overhead_us, out_wcrt, out_sched);
+  // Nothing in the array has to be cleared first: the plan kernels write the header (counts,
+  // starts, zeroed work counters), every per-block count and every permutation entry that the
+  // analysis kernels of this call read.
+  return enqueue_batch(p, g_static_scratch_ptr[dev], (size_t)GCAPS_RTA_STATIC_SCRATCH_BYTES,
+                       di.sm_count, (cudaStream_t)stream);
 }
 
 int gcaps_rta_validate(const gcaps_tasksets_t *ts, int64_t n_tasksets, int32_t *out_err,
@@ -793,6 +837,8 @@ const char *gcaps_rta_strerror(int code) {
     case GCAPS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case GCAPS_ERR_CUDA: return "CUDA runtime error (see gcaps_rta_last_cuda_error)";
     case GCAPS_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+    case GCAPS_ERR_TOO_LARGE:
+      return "batch exceeds GCAPS_RTA_STATIC_MAX_TASKSETS: split it or use gcaps_rta_batch";
     default: return "unknown error code";
   }
 }
