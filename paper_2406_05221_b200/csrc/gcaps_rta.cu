@@ -1,18 +1,25 @@
 // gcaps_rta.cu -- batched worst-case response-time analysis of GPU-using real-time tasksets
 // (GCAPS, ECRTS 2024, arXiv 2406.05221, Sec. 6) for NVIDIA B200 (sm_100a).
 //
-// One group of LPT lanes (a warp or a slice of one) analyses one taskset at a time:
-//   stage      coalesced loads of the taskset's per-task slices; per-task sums over its segments
-//              (C_i, G^m_i, G^e_i, RR slice count of Eq. 3) go to shared memory in priority order
-//   order      rank of every task by (priority desc, position asc)
-//   iterate    for each task in that order the recurrence of Eq. 1 with the lemma set of the
+// One warp analyses one taskset at a time:
+//   stage      coalesced loads of the taskset's per-task slices into registers (lane = task)
+//   aggregate  coalesced loads of the segment arrays, warp prefix sums into shared memory; the
+//              per-task sums C_i, G^m_i, G^e_i and the RR slice count of Eq. 3 are differences of
+//              two prefix values
+//   order      rank of every task by (priority desc, position asc); the per-task values move
+//              through shared memory to the lane that owns the task's rank
+//   iterate    for each task in rank order the recurrence of Eq. 1 with the lemma set of the
 //              chosen analysis: lanes over the higher-priority interferers, each evaluating
-//              ceil((R+J)/T_h)*W terms, summed across the group with __shfl_xor
-//   publish    R_i feeds the jitters J^c, J^g of later tasks; first deadline miss ends the taskset
-//   write      out_wcrt through shared memory (coalesced), out_sched one byte
-// Tasksets are binned by size (a small plan pass writes a permutation into the caller's
-// workspace) so that groups of a launch see similar amounts of work; inside a launch groups pull
-// chunks of tasksets from a counter, because iteration counts differ widely.
+//              ceil((R+J)/T_h)*W terms (division by the invariant T_h is a multiply-high by a
+//              per-task reciprocal), summed across the warp
+//   publish    the lane that owns the converged task keeps R_i and forms its jitters J^c, J^g
+//   early exit the first deadline miss ends the taskset
+//   write      out_wcrt (one value per task), out_sched (one byte per taskset)
+// The fast path holds every time in 32 bits and is taken when all values of a taskset are below
+// 2^26 us; any other taskset goes through an exact 64-bit path with saturating arithmetic.
+// Tasksets are binned by size (a small plan pass writes a permutation into the workspace) so that
+// the warps of a launch hold the same number of tasks per lane; inside a launch warps pull chunks
+// of tasksets from a counter, because iteration counts differ widely.
 //
 // Everything is integer arithmetic on microseconds.  No tensor cores: nothing here is a dense
 // contraction.  No host synchronisation and no allocation in gcaps_rta_batch.
@@ -29,10 +36,10 @@ typedef unsigned long long u64;
 typedef long long i64;
 
 constexpr int kNumBins = 6;
-// largest taskset size of each bin and the lanes that cooperate on one taskset of it
-__host__ __device__ constexpr int bin_max_n(int b) {
-  return b == 0 ? 8 : b == 1 ? 16 : b == 2 ? 32 : b == 3 ? 64 : b == 4 ? 96 : GCAPS_RTA_MAX_TASKS;
-}
+typedef unsigned int u32;
+// size bins: at most 32, 64, 96, 128, 192, 256 tasks = 1, 2, 3, 4, 6, 8 tasks per lane
+constexpr u32 kFastLimit = 1u << 26;  // fast path: every time of the taskset is below this
+constexpr u32 kFastClamp = 1u << 26;  // ... so a sum clamped here still exceeds every deadline
 constexpr int kBlockThreads = 128;
 constexpr int kPlanItems = 1024;  // tasksets per plan block
 constexpr u64 kClamp = 1ull << 50;  // any quantity >= 2^50 exceeds every deadline (<= 2^40)
@@ -53,6 +60,9 @@ struct KParams {
   i64 n_tasksets;
   int policy;  // GCAPS_POLICY_* | flags
   i64 L, ovh;
+  // division by L in the 32-bit path: 0 = multiply-high by l_magic then shift, 1 = L is 1,
+  // 2 = L >= 2^26 (every non-empty pure GPU part takes one slice)
+  u32 l_mode, l_magic, l_shift;
   i64 *out_wcrt;
   uint8_t *out_sched;
   PlanHeader *hdr;
@@ -61,11 +71,11 @@ struct KParams {
 };
 
 __device__ __forceinline__ int size_bin(i64 n) {
-  if (n <= 8) return 0;  // also negative / broken ranges: rejected by the analysis kernel
-  if (n <= 16) return 1;
-  if (n <= 32) return 2;
-  if (n <= 64) return 3;
-  if (n <= 96) return 4;
+  if (n <= 32) return 0;  // also negative / broken ranges: rejected by the analysis kernel
+  if (n <= 64) return 1;
+  if (n <= 96) return 2;
+  if (n <= 128) return 3;
+  if (n <= 192) return 4;
   if (n <= GCAPS_RTA_MAX_TASKS) return 5;
   return 0;
 }
@@ -364,29 +374,412 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
   __syncwarp(mask);
 }
 
-// Persistent launch over one size bin: groups pull chunks of tasksets from the bin's counter.
-template <int LPT, int MAXN>
-__global__ void __launch_bounds__(kBlockThreads) rta_bin_kernel(KParams p, int bin) {
+// ---------------------------------------------------------------------------------------------
+// 32-bit fast path
+// ---------------------------------------------------------------------------------------------
+constexpr unsigned int kFull = 0xffffffffu;
+
+__device__ __forceinline__ u32 warp_incl_scan(u32 x, int lane) {
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 y = __shfl_up_sync(kFull, x, d);
+    if (lane >= d) x += y;
+  }
+  return x;
+}
+
+// Reciprocal of a divisor d in [2, 2^26): floor(x / d) = umulhi(x, magic) >> shift for every
+// x < 2^28.  With s = ceil(log2 d) and k = max(28 + s, 32), magic = ceil(2^k / d) < 2^32 and its
+// error magic*d - 2^k < d <= 2^s, so x * error < 2^k and the quotient is exact.
+__host__ __device__ __forceinline__ void make_reciprocal(u32 d, u32 &magic, u32 &shift) {
+#ifdef __CUDA_ARCH__
+  const int s = 32 - __clz((int)(d - 1));
+#else
+  int s = 0;
+  while ((1u << s) < d) ++s;
+#endif
+  const int k = (28 + s) > 32 ? (28 + s) : 32;
+  shift = (u32)(k - 32);
+#ifdef __CUDA_ARCH__
+  // estimate 2^k / d in double precision (error far below 1), then make it exact with integers
+  const double two_k = __hiloint2double((1023 + k) << 20, 0);
+  u32 q = __double2uint_rd(two_k * __drcp_rn((double)d));
+  i64 rem = (i64)(1ull << k) - (i64)((u64)q * d);
+  if (rem < 0) {
+    q -= 1;
+    rem += d;
+  } else if (rem >= (i64)d) {
+    q += 1;
+    rem -= d;
+  }
+  magic = rem == 0 ? q : q + 1;
+#else
+  const u64 two_k = 1ull << k;
+  magic = (u32)((two_k + d - 1) / d);
+#endif
+}
+
+// Exclusive prefix sums of X[0..N) into P[0..N] (32-bit).  `ok` drops if an element is outside
+// [0, 2^26).  Needs N <= capacity of P - 1.
+__device__ __forceinline__ void scan_one(const i64 *__restrict__ X, int N, u32 *P, int lane, bool &ok) {
+  u32 carry = 0;
+  if (lane == 0) P[0] = 0;
+  for (int e0 = 0; e0 < N; e0 += 32) {
+    const int e = e0 + lane;
+    const i64 v = e < N ? X[e] : 0;
+    ok &= (u64)v < kFastLimit;
+    const u32 x = warp_incl_scan((u32)v, lane) + carry;
+    if (e < N) P[e + 1] = x;
+    carry = __shfl_sync(kFull, x, 31);
+  }
+}
+
+// MODE: 0 GCAPS self-suspension, 1 GCAPS busy-waiting, 2 RR self-suspension, 3 RR busy-waiting.
+// Returns false, having written nothing, if the taskset is not eligible for 32-bit arithmetic
+// (or is invalid): the caller then runs the exact 64-bit path, which also does the validation.
+template <int SLOTS, int MODE>
+__device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane) {
+  constexpr int MAXN = 32 * SLOTS;
+  constexpr int CAP = 10 * MAXN;  // elements one prefix buffer can take
+  constexpr bool kGcaps = MODE < 2;
+  const bool literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
+  u32 *P0 = buf, *P1 = buf + CAP + 32;
+
+  // ---- stage: per-task scalars, lane = position -------------------------------------------
+  const i64 cfirst = p.cseg_off[a] - p.cseg_base, gfirst = p.gseg_off[a] - p.gseg_base;
+  const i64 Nc64 = p.cseg_off[a + n] - p.cseg_base - cfirst;
+  const i64 Ng64 = p.gseg_off[a + n] - p.gseg_base - gfirst;
+  if (cfirst < 0 || Nc64 < 0 || cfirst + Nc64 > p.n_csegs || Nc64 > CAP || gfirst < 0 || Ng64 < 0 ||
+      gfirst + Ng64 > p.n_gsegs || Ng64 > CAP)
+    return false;
+  const int Nc = (int)Nc64, Ng = (int)Ng64;
+  u32 T[SLOTS], D[SLOTS], core[SLOTS];
+  int prio[SLOTS], c0[SLOTS], g0[SLOTS];
+  bool ok = true, prio_small = true;
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int i = lane + 32 * s;
+    const bool v = i < n;
+    const i64 k = a + (v ? i : 0);
+    const i64 t64 = p.period[k], d64 = p.deadline[k], pr = p.priority[k], c64 = p.core[k];
+    const i64 co = p.cseg_off[k] - p.cseg_base - cfirst, go = p.gseg_off[k] - p.gseg_base - gfirst;
+    ok &= !v || ((u64)(t64 - 2) < (u64)(kFastLimit - 2) && d64 >= 1 && d64 <= t64 &&
+                 (u64)c64 <= (u64)GCAPS_RTA_MAX_CORE && (u64)co <= (u64)Nc && (u64)go <= (u64)Ng);
+    prio_small &= !v || pr == (i64)(int)pr;
+    T[s] = v ? (u32)t64 : 2u;
+    D[s] = (u32)d64;
+    core[s] = (u32)c64;
+    prio[s] = v ? (int)pr : (int)0x80000000;
+    c0[s] = v ? (int)co : Nc;
+    g0[s] = v ? (int)go : Ng;
+  }
+  // end offsets: the next task's start (positions beyond n hold the total)
+  int c1[SLOTS], g1[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int cn = __shfl_down_sync(kFull, c0[s], 1), gn = __shfl_down_sync(kFull, g0[s], 1);
+    const int ch = __shfl_sync(kFull, s + 1 < SLOTS ? c0[s + 1 < SLOTS ? s + 1 : s] : Nc, 0);
+    const int gh = __shfl_sync(kFull, s + 1 < SLOTS ? g0[s + 1 < SLOTS ? s + 1 : s] : Ng, 0);
+    c1[s] = lane == 31 ? ch : cn;
+    g1[s] = lane == 31 ? gh : gn;
+    ok &= (u32)(c1[s] - c0[s]) < 64u && (u32)(g1[s] - g0[s]) < 64u;
+  }
+  if (!__all_sync(kFull, ok)) return false;
+
+  // ---- aggregate: prefix sums of the segment arrays, per-task sums as differences ---------
+  u32 A[SLOTS], Ge[SLOTS], S[SLOTS];  // C+G^m, G^e, and 2*eps*eta (GCAPS) or (L+theta)*slices (RR)
+  scan_one(p.cseg_wcet + cfirst, Nc, P0, lane, ok);
+  __syncwarp();
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) A[s] = P0[c1[s]] - P0[c0[s]];
+  __syncwarp();
+  {  // G^m into P0 and G^e into P1, interleaved
+    const i64 *__restrict__ Xm = p.gseg_misc + gfirst, *__restrict__ Xe = p.gseg_exec + gfirst;
+    u32 cm = 0, ce = 0;
+    if (lane == 0) P0[0] = 0, P1[0] = 0;
+    for (int e0 = 0; e0 < Ng; e0 += 32) {
+      const int e = e0 + lane;
+      const i64 vm = e < Ng ? Xm[e] : 0, ve = e < Ng ? Xe[e] : 0;
+      ok &= (u64)vm < kFastLimit && (u64)ve < kFastLimit;
+      u32 xm = (u32)vm, xe = (u32)ve;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const u32 ym = __shfl_up_sync(kFull, xm, d), ye = __shfl_up_sync(kFull, xe, d);
+        if (lane >= d) xm += ym, xe += ye;
+      }
+      xm += cm, xe += ce;
+      if (e < Ng) P0[e + 1] = xm, P1[e + 1] = xe;
+      cm = __shfl_sync(kFull, xm, 31), ce = __shfl_sync(kFull, xe, 31);
+    }
+  }
+  __syncwarp();
+  u32 eta[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const u32 C = A[s], Gm = P0[g1[s]] - P0[g0[s]];
+    Ge[s] = P1[g1[s]] - P1[g0[s]];
+    eta[s] = (u32)(g1[s] - g0[s]);
+    A[s] = C + Gm;
+    ok &= C < kFastLimit && Gm < kFastLimit && Ge[s] < kFastLimit && A[s] < kFastLimit;
+  }
+  __syncwarp();
+  if (!kGcaps) {  // Eq. 3: slices of every pure GPU part, summed per task
+    const i64 *__restrict__ Xe = p.gseg_exec + gfirst;
+    u32 carry = 0;
+    if (lane == 0) P0[0] = 0;
+    for (int e0 = 0; e0 < Ng; e0 += 32) {
+      const int e = e0 + lane;
+      const u32 ve = e < Ng ? (u32)Xe[e] : 0u;  // range was checked by the pass above
+      u32 sl;
+      if (p.l_mode == 0) sl = __umulhi(ve + (u32)p.L - 1u, p.l_magic) >> p.l_shift;
+      else if (p.l_mode == 1) sl = ve;
+      else sl = ve > 0 ? 1u : 0u;
+      const u32 x = warp_incl_scan(sl, lane) + carry;
+      if (e < Ng) P0[e + 1] = x;
+      carry = __shfl_sync(kFull, x, 31);
+    }
+    __syncwarp();
+  }
+  // ---- constants of Eq. 1 that do not depend on R ------------------------------------------
+  int n_gpu = 0;  // N_g
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(kFull, eta[s] > 0));
+  u32 base[SLOTS];
+  const u64 ovh = (u64)p.ovh;
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    u64 b64;
+    if (kGcaps) {
+      const u64 star = 2 * ovh * eta[s];  // eta < 64, ovh <= 2^40
+      ok &= star < kFastLimit;
+      S[s] = (u32)star;
+      b64 = (u64)A[s] + Ge[s] + star + ((u64)eta[s] + 1) * ovh;  // C_i + G*_i + B^C_i
+    } else {
+      const u64 slices = P0[g1[s]] - P0[g0[s]];
+      const u64 lt = (u64)p.L + ovh;  // <= 2^41
+      u64 B = slices == 0 ? 0 : (lt >= kFastClamp ? kFastClamp : lt * slices);  // < 2^26 * 2^32
+      if (B > kFastClamp) B = kFastClamp;
+      S[s] = (u32)B;
+      u64 ie = eta[s] > 0 ? B * (u64)(n_gpu - 1) : 0;  // Lemma 1
+      b64 = (u64)A[s] + Ge[s] + ie;
+    }
+    base[s] = b64 > (u64)(2 * kFastClamp) ? 2 * kFastClamp : (u32)b64;
+  }
+  if (!__all_sync(kFull, ok)) return false;
+  __syncwarp();
+
+  // ---- order ---------------------------------------------------------------------------------
+  int rank[SLOTS];
+  bool dense = __all_sync(kFull, prio_small);
+  if (dense) {  // distinct priorities max-n+1 .. max: the rank is max - priority
+    int m = prio[0];
+#pragma unroll
+    for (int s = 1; s < SLOTS; ++s) m = prio[s] > m ? prio[s] : m;
+    const int pmax = __reduce_max_sync(kFull, m);
+    bool in = true;
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const i64 r = (i64)pmax - (i64)prio[s];
+      const bool v = lane + 32 * s < n;
+      in &= !v || r < (i64)n;
+      rank[s] = v ? (int)r : 0;
+    }
+    dense = __all_sync(kFull, in);
+    if (dense) {
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s)
+        if (lane + 32 * s < n) buf[rank[s]] = (u32)(lane + 32 * s);
+      __syncwarp();
+      bool uniq = true;
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s)
+        if (lane + 32 * s < n) uniq &= buf[rank[s]] == (u32)(lane + 32 * s);
+      dense = __all_sync(kFull, uniq);
+      __syncwarp();
+    }
+  }
+  if (!dense) {  // any priorities: count the tasks that come before
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const int i = lane + 32 * s;
+      const i64 pi = p.priority[a + (i < n ? i : 0)];
+      int r = 0;
+      for (int q = 0; q < n; ++q) {
+        const i64 pq = p.priority[a + q];
+        r += (pq > pi || (pq == pi && q < i)) ? 1 : 0;
+      }
+      rank[s] = r;
+    }
+  }
+  // ---- move the per-task values to the lane that owns the rank -----------------------------
+  // word w of rank r sits at buf[w * MAXN + r]; words 1, 2, 6, 7 are read again per task below
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int i = lane + 32 * s;
+    if (i < n) {
+      const int r = rank[s];
+      buf[0 * MAXN + r] = T[s];
+      buf[1 * MAXN + r] = D[s];
+      buf[2 * MAXN + r] = base[s];
+      buf[3 * MAXN + r] = A[s];
+      buf[4 * MAXN + r] = Ge[s];
+      buf[5 * MAXN + r] = S[s];
+      buf[6 * MAXN + r] = core[s];
+      buf[7 * MAXN + r] = (u32)i | (eta[s] > 0 ? 0x10000u : 0u);
+    }
+  }
+  __syncwarp();
+  u32 magic[SLOTS], shift[SLOTS], Tm1[SLOTS], pos_of[SLOTS];
+  bool gpu[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int r = lane + 32 * s;
+    const bool v = r < n;
+    const u32 Tr = v ? buf[0 * MAXN + r] : 2u;
+    A[s] = v ? buf[3 * MAXN + r] : 0u;
+    Ge[s] = v ? buf[4 * MAXN + r] : 0u;
+    S[s] = v ? buf[5 * MAXN + r] : 0u;
+    core[s] = v ? buf[6 * MAXN + r] : 0xffffffffu;
+    const u32 meta = v ? buf[7 * MAXN + r] : 0u;
+    pos_of[s] = meta & 0xffffu;
+    gpu[s] = (meta & 0x10000u) != 0;
+    Tm1[s] = Tr - 1;
+    make_reciprocal(Tr, magic[s], shift[s]);
+  }
+
+  // ---- iterate in rank order ------------------------------------------------------------------
+  u32 Jc[SLOTS], Jg[SLOTS], Rown[SLOTS];  // jitters with T_h - 1 folded in (ceiling), own result
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Rown[s] = 0;
+  int n_done = n;
+  i64 verdict = 0;
+  for (int pos = 0; pos < n; ++pos) {
+    const u32 Di = buf[1 * MAXN + pos], base_i = buf[2 * MAXN + pos], core_i = buf[6 * MAXN + pos];
+    const bool gi = (buf[7 * MAXN + pos] & 0x10000u) != 0;
+    u32 nu = 0;
+    if (MODE == 3) {  // Lemma 4: N_g - |{h in hpp(i): GPU-using}| + 1
+      int c = 0;
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s)
+        c += __popc(__ballot_sync(kFull, lane + 32 * s < pos && core[s] == core_i && gpu[s]));
+      nu = (u32)(n_gpu - c + 1);
+    }
+    // the (J, W) pairs of this task's interferers; W = 0 where a pair does not apply
+    u32 J1[SLOTS], W1[SLOTS], J2[SLOTS], W2[SLOTS];
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const bool act = lane + 32 * s < pos;
+      const bool same = core[s] == core_i, gh = gpu[s];
+      u32 w1 = 0, w2 = 0, j1 = Tm1[s], j2 = Tm1[s];
+      if (MODE == 0) {
+        if (same) {  // Lemma 15
+          w1 = A[s] + (gh ? S[s] : 0u);
+          j1 = gh ? Jc[s] : Tm1[s];
+          if (gh && gi) w2 = Ge[s], j2 = Jg[s];  // Lemma 13, same core
+        } else if (gh && gi) {
+          w1 = Ge[s] + S[s], j1 = Jg[s];  // Lemma 13, other cores
+        }
+      } else if (MODE == 1) {
+        if (same) {
+          w1 = A[s] + ((gh && (gi || !literal)) ? Ge[s] + S[s] : 0u);  // Lemmas 12, 10
+        } else if (gh) {
+          w1 = Ge[s] + S[s], j1 = Jg[s];  // Lemma 10 / Lemma 11
+        }
+      } else if (MODE == 2) {
+        if (same) w1 = A[s], j1 = (gh || literal) ? Jc[s] : Tm1[s];  // Lemma 7
+      } else {
+        if (same) {  // Lemmas 5 and 4
+          const u64 w = (u64)A[s] + (gh ? (u64)S[s] * nu : 0ull);
+          w1 = w > kFastClamp ? kFastClamp : (u32)w;
+        }
+      }
+      J1[s] = j1, W1[s] = act ? w1 : 0u, J2[s] = j2, W2[s] = act ? w2 : 0u;
+    }
+    const int smax = pos == 0 ? -1 : (pos - 1) >> 5;
+    u32 R = base_i;
+    i64 v = 0;
+    i64 sweeps = 0;
+    for (;;) {
+      if (R > Di) {
+        v = GCAPS_WCRT_MISS;
+        break;
+      }
+      if (sweeps >= GCAPS_RTA_ITER_CAP) {
+        v = GCAPS_WCRT_ITER_LIMIT;
+        break;
+      }
+      sweeps += 1;
+      u64 acc = 0;
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s) {
+        if (s <= smax) {
+          acc += (u64)(__umulhi(R + J1[s], magic[s]) >> shift[s]) * W1[s];
+          if (MODE == 0) acc += (u64)(__umulhi(R + J2[s], magic[s]) >> shift[s]) * W2[s];
+        }
+      }
+      const u32 part = acc > (u64)kFastClamp ? kFastClamp : (u32)acc;
+      const u32 next = base_i + __reduce_add_sync(kFull, part);
+      if (next == R) break;
+      R = next;
+    }
+    if (v != 0) {
+      n_done = pos;
+      verdict = v;
+      break;
+    }
+    // publish: the owner of this rank keeps R_i and its jitters J^c = R - (C+G^m), J^g = R - G^e
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      if (lane + 32 * s == pos) {
+        Rown[s] = R;
+        Jc[s] = R - A[s] + Tm1[s];
+        Jg[s] = R - Ge[s] + Tm1[s];
+      }
+    }
+  }
+  // ---- write ----------------------------------------------------------------------------------
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int r = lane + 32 * s;
+    if (r < n)
+      p.out_wcrt[a + pos_of[s]] = r < n_done ? (i64)Rown[s] : (r == n_done ? verdict : (i64)GCAPS_WCRT_SKIPPED);
+  }
+  if (lane == 0) p.out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
+  __syncwarp();
+  return true;
+}
+
+// shared memory of one warp, in 32-bit words: two prefix buffers of 10*MAXN+32 words each; the
+// image of the exact path (GroupSmem, 74 bytes per task) fits in the same space
+template <int SLOTS>
+__host__ __device__ constexpr int warp_words() { return 20 * 32 * SLOTS + 64; }
+
+// Persistent launch over one size bin: warps pull chunks of tasksets from the bin's counter.
+template <int SLOTS, int MODE>
+__global__ void __launch_bounds__(kBlockThreads) rta_kernel(KParams p, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  constexpr int kGroupsPerWarp = 32 / LPT;
-  constexpr int kChunk = 4;  // tasksets per group per pull
-  GroupSmem<MAXN> *all = reinterpret_cast<GroupSmem<MAXN> *>(smem_raw);
-  const int warp_in_block = threadIdx.x >> 5, lane32 = threadIdx.x & 31;
-  const int group_in_warp = lane32 / LPT, lane = lane32 % LPT;
-  GroupSmem<MAXN> &s = all[warp_in_block * kGroupsPerWarp + group_in_warp];
-  const unsigned int mask =
-      LPT == 32 ? 0xffffffffu : (((1u << LPT) - 1u) << (group_in_warp * LPT));
+  constexpr int MAXN = 32 * SLOTS;
+  constexpr int kChunk = 4;  // tasksets per pull
+  static_assert(sizeof(GroupSmem<MAXN>) <= sizeof(u32) * warp_words<SLOTS>(), "exact path fits");
+  const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * warp_words<SLOTS>();
   const unsigned int start = p.hdr->bin_start[bin], count = p.hdr->bin_count[bin];
   for (;;) {
     unsigned int first = 0;
-    if (lane32 == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)(kChunk * kGroupsPerWarp));
-    first = __shfl_sync(0xffffffffu, first, 0);
+    if (lane == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
+    first = __shfl_sync(kFull, first, 0);
     if (first >= count) break;
-    for (int c = 0; c < kChunk; ++c) {
-      const unsigned int idx = first + c * kGroupsPerWarp + group_in_warp;
-      if (idx < count) analyse_taskset<LPT, MAXN>(p, (i64)p.perm[start + idx], s, lane, mask);
+    const unsigned int last = first + kChunk < count ? first + kChunk : count;
+    for (unsigned int idx = first; idx < last; ++idx) {
+      const i64 t = (i64)p.perm[start + idx];
+      const i64 a = p.task_off[t] - p.task_base, b = p.task_off[t + 1] - p.task_base;
+      bool done = false;
+      if (a >= 0 && b > a && b <= p.n_tasks && b - a <= MAXN)
+        done = analyse_fast<SLOTS, MODE>(p, t, a, (int)(b - a), buf, lane);
+      __syncwarp();
+      if (!done) analyse_taskset<32, MAXN>(p, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, kFull);
+      __syncwarp();
     }
-    __syncwarp();
   }
 }
 
@@ -501,35 +894,55 @@ void fill_params(KParams *p, const gcaps_tasksets_t *ts, int64_t n_tasksets, int
   p->policy = policy;
   p->L = (policy & 0xff) == GCAPS_POLICY_RR ? L : 1;
   p->ovh = ovh;
+  if (p->L == 1) {
+    p->l_mode = 1;
+  } else if (p->L >= (i64)kFastLimit) {
+    p->l_mode = 2;
+  } else {
+    p->l_mode = 0;
+    make_reciprocal((u32)p->L, p->l_magic, p->l_shift);
+  }
   p->out_wcrt = (i64 *)out_wcrt;
   p->out_sched = out_sched;
 }
 
-template <int LPT, int MAXN>
+template <int SLOTS, int MODE>
 cudaError_t launch_bin(const KParams &p, int bin, int sm_count, cudaStream_t st) {
-  constexpr int kGroups = kBlockThreads / LPT;
-  const size_t smem = sizeof(GroupSmem<MAXN>) * kGroups;
-  static bool attr_done[64] = {false};
+  constexpr int kWarps = kBlockThreads / 32;
+  const size_t smem = sizeof(u32) * warp_words<SLOTS>() * kWarps;
+  static int blocks_per_sm[64] = {0};  // per device; 0 = not set up yet
   int dev = 0;
-  cudaGetDevice(&dev);
-  if (!attr_done[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(rta_bin_kernel<LPT, MAXN>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_done[dev & 63] = true;
-  }
-  int per_sm = 1;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-      &per_sm, rta_bin_kernel<LPT, MAXN>, kBlockThreads, smem);
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (per_sm < 1) per_sm = 1;
-  // never more blocks than the bin could feed (the exact bin population lives on the device)
-  long long want = (p.n_tasksets + kGroups - 1) / kGroups;
-  long long grid = (long long)sm_count * per_sm;
+  dev &= 63;
+  if (blocks_per_sm[dev] == 0) {
+    e = cudaFuncSetAttribute(rta_kernel<SLOTS, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 1;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rta_kernel<SLOTS, MODE>,
+                                                      kBlockThreads, smem);
+    if (e != cudaSuccess) return e;
+    blocks_per_sm[dev] = per_sm < 1 ? 1 : per_sm;
+  }
+  // never more warps than the bin could feed (the exact bin population lives on the device)
+  long long want = (p.n_tasksets + kWarps - 1) / kWarps;
+  long long grid = (long long)sm_count * blocks_per_sm[dev];
   if (grid > want) grid = want;
   if (grid < 1) grid = 1;
-  rta_bin_kernel<LPT, MAXN><<<(unsigned int)grid, kBlockThreads, smem, st>>>(p, bin);
+  rta_kernel<SLOTS, MODE><<<(unsigned int)grid, kBlockThreads, smem, st>>>(p, bin);
   return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t launch_all_bins(const KParams &p, int sm_count, cudaStream_t st) {
+  cudaError_t e = launch_bin<1, MODE>(p, 0, sm_count, st);
+  if (e == cudaSuccess) e = launch_bin<2, MODE>(p, 1, sm_count, st);
+  if (e == cudaSuccess) e = launch_bin<3, MODE>(p, 2, sm_count, st);
+  if (e == cudaSuccess) e = launch_bin<4, MODE>(p, 3, sm_count, st);
+  if (e == cudaSuccess) e = launch_bin<6, MODE>(p, 4, sm_count, st);
+  if (e == cudaSuccess) e = launch_bin<8, MODE>(p, 5, sm_count, st);
+  return e;
 }
 
 int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_count, cudaStream_t st) {
@@ -546,12 +959,13 @@ int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_cou
   plan_scan_kernel<<<1, 1024, 0, st>>>(p, (unsigned int)nb);
   plan_scatter_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
   cudaError_t e = cudaGetLastError();
-  if (e == cudaSuccess) e = launch_bin<8, 8>(p, 0, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<16, 16>(p, 1, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<32, 32>(p, 2, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<32, 64>(p, 3, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<32, 96>(p, 4, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<32, GCAPS_RTA_MAX_TASKS>(p, 5, sm_count, st);
+  if (e == cudaSuccess) {
+    const bool rr = (p.policy & 0xff) == GCAPS_POLICY_RR, busy = (p.policy & GCAPS_RTA_BUSY) != 0;
+    if (!rr && !busy) e = launch_all_bins<0>(p, sm_count, st);
+    else if (!rr) e = launch_all_bins<1>(p, sm_count, st);
+    else if (!busy) e = launch_all_bins<2>(p, sm_count, st);
+    else e = launch_all_bins<3>(p, sm_count, st);
+  }
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     return GCAPS_ERR_CUDA;

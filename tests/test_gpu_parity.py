@@ -178,6 +178,40 @@ def test_iteration_cap_and_extreme_values():
     assert w[1] == binding.WCRT_ITER_LIMIT and w[3] == binding.WCRT_MISS
 
 
+def test_values_around_the_32_bit_path_limit():
+    """Tasksets whose times sit just below, at and above 2^26 us (where the kernels switch from
+    32-bit to exact 64-bit arithmetic), mixed in one batch; also small periods down to 2 and 1,
+    priorities that are dense, sparse, negative, huge or tied, and tasks with many segments."""
+    rng = np.random.default_rng(21)
+    lim = 1 << 26
+    sets = []
+    for top in (lim - 1, lim, lim + 1, 3 * lim, lim // 2):
+        for n in (3, 20, 33, 70):
+            ts = []
+            for i in range(n):
+                T = int(top if i % 3 == 0 else rng.integers(top // 8, top))
+                ng = int(rng.integers(0, 3))
+                ts.append(dict(T=T, D=T - int(rng.integers(0, 3)), prio=0, core=int(rng.integers(0, 4)),
+                               cseg=[int(rng.integers(0, T // (8 * n) + 2)) for _ in range(ng + 1)],
+                               gseg=[(int(rng.integers(0, T // (16 * n) + 2)), int(rng.integers(0, T // (10 * n) + 2)))
+                                     for _ in range(ng)]))
+            style = len(sets) % 5
+            for i, tk in enumerate(ts):
+                tk["prio"] = [n - i, 1000 * (n - i) - 7, -(i + 1), (1 << 40) + (n - i), (n - i) // 3][style]
+            sets.append(ts)
+    # tiny periods, and one task with 70 segments of each kind (beyond the per-task fast limit)
+    sets.append([dict(T=2, prio=3, core=0, cseg=[1]), dict(T=3, prio=2, core=0, cseg=[1]),
+                 dict(T=40, prio=1, core=0, cseg=[1], gseg=[(0, 1)])])
+    sets.append([dict(T=1, prio=3, core=0, cseg=[1]), dict(T=7, prio=2, core=0, cseg=[1])])
+    sets.append([dict(T=100000, prio=2, core=0, cseg=[3] * 71, gseg=[(1, 2)] * 70),
+                 dict(T=200000, prio=1, core=0, cseg=[5], gseg=[(1, 7)])])
+    sets.append([dict(T=50000 + i, prio=i, core=i % 3, cseg=[2] * 12, gseg=[(1, 1)] * 11) for i in range(30)])
+    b = batch_of(sets)
+    for policy in ALL_MODES:
+        for L, ovh in ((1024, 50), (1, 0), (lim, 1), (lim - 1, lim - 1), (3, 1 << 21)):
+            assert_parity(b, policy, L, ovh, "limit L=%d ovh=%d" % (L, ovh))
+
+
 def test_determinism_and_output_reuse():
     b = taskgen.WORKLOADS["divergence"].generate(1000, 4000)
     ts = binding.DeviceTasksets.from_host(b)
