@@ -32,6 +32,8 @@ def build_cuda(force: bool = False, verbose: bool = False) -> str:
     """Compiles csrc/gcaps_rta.cu for sm_100a into libgcaps_rta.so beside this file."""
     if force or cuda_lib_is_stale():
         tmp = CUDA_LIB + ".%d.tmp" % os.getpid()
+        if os.path.exists(CUDA_LIB):
+            os.remove(CUDA_LIB)  # a failed build must not leave an older library behind
         cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp, CUDA_SRC]
         subprocess.check_call(cmd)
         os.replace(tmp, CUDA_LIB)

@@ -191,7 +191,6 @@ struct GroupSmem {
   u64 T[MAXN];     // period
   u64 D[MAXN];     // deadline
   u64 A[MAXN];     // C + G^m
-  u64 Cc[MAXN];    // C
   u64 Ge[MAXN];    // G^e
   u64 Star[MAXN];  // 2 * eps * eta^g   (GCAPS)   /   (L + theta) * slices, clamped   (RR)
   u64 R[MAXN];     // converged response time
@@ -269,7 +268,6 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
     s.T[rank] = (u64)p.period[k];
     s.D[rank] = (u64)p.deadline[k];
     s.A[rank] = C + Gm;
-    s.Cc[rank] = C;
     s.Ge[rank] = Ge;
     s.Star[rank] = policy == GCAPS_POLICY_GCAPS ? 2 * ovh * (u64)eta : sat_mul(L + ovh, slices);
     s.core[rank] = (int)p.core[k];
@@ -329,7 +327,7 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
         const u64 Jc = Rh - s.A[h], Jg = Rh - s.Ge[h];
         u64 term = 0;
         if (policy == GCAPS_POLICY_GCAPS && !busy) {
-          if (same && !gh) term = sat_mul(ceil_div64(R, Th), s.Cc[h]);             // Lemma 15
+          if (same && !gh) term = sat_mul(ceil_div64(R, Th), s.A[h]);  // Lemma 15 (G^m_h = 0)
           if (same && gh) term = sat_mul(ceil_div64(R + Jc, Th), s.A[h] + s.Star[h]);
           if (same && gh && gi) term += sat_mul(ceil_div64(R + Jg, Th), s.Ge[h]);   // Lemma 13
           if (!same && gh && gi) term = sat_mul(ceil_div64(R + Jg, Th), s.Ge[h] + s.Star[h]);
@@ -419,59 +417,237 @@ __host__ __device__ __forceinline__ void make_reciprocal(u32 d, u32 &magic, u32 
 #endif
 }
 
-// Exclusive prefix sums of X[0..N) into P[0..N] (32-bit).  `ok` drops if an element is outside
-// [0, 2^26).  Needs N <= capacity of P - 1.
-__device__ __forceinline__ void scan_one(const i64 *__restrict__ X, int N, u32 *P, int lane, bool &ok) {
-  u32 carry = 0;
-  if (lane == 0) P[0] = 0;
-  for (int e0 = 0; e0 < N; e0 += 32) {
-    const int e = e0 + lane;
-    const i64 v = e < N ? X[e] : 0;
-    ok &= (u64)v < kFastLimit;
-    const u32 x = warp_incl_scan((u32)v, lane) + carry;
-    if (e < N) P[e + 1] = x;
-    carry = __shfl_sync(kFull, x, 31);
+// ---- running sums of a segment array, 128 elements per step ------------------------------------
+// Lane l takes four consecutive elements (two 16-byte loads), so a warp reads 1 KB contiguous.
+// Loads must start on a 16-byte boundary: when the slice starts on an odd element the step begins
+// one element early (`par` = 1).  Q[x] receives the sum (modulo 2^32) of elements -par .. x - par;
+// Q[-1] is a guard word holding 0.  For 0 <= lo <= hi <= N the sum of elements [lo, hi) is
+// Q[hi - 1 + par] - Q[lo - 1 + par]: a borrowed element in front only shifts every entry by the
+// same amount, and elements behind the slice only reach entries that are never read.
+struct Quad {
+  i64 v[4];
+};
+
+// Elements e .. e+3 of X, for a slice whose 16-byte pairs all lie inside the array (the common
+// case, checked once per taskset by the caller).  Pairs that start at or behind N are not read.
+__device__ __forceinline__ void load_quad_inside(const i64 *__restrict__ X, int e, int N, Quad &q) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    longlong2 w = make_longlong2(0, 0);
+    if (e + 2 * h < N) w = __ldg(reinterpret_cast<const longlong2 *>(X + e + 2 * h));
+    q.v[2 * h] = w.x, q.v[2 * h + 1] = w.y;
+  }
+}
+
+// The same for a slice at the very edge of its array: only wanted elements inside [lo, hi) are
+// touched, everything else reads as 0.
+__device__ __noinline__ Quad load_quad_edge(const i64 *__restrict__ X, int e, int N, const i64 *lo,
+                                            const i64 *hi) {
+  Quad q;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const i64 *ptr = X + e + j;
+    q.v[j] = (e + j >= 0 && e + j < N && ptr >= lo && ptr < hi) ? __ldg(ptr) : 0;
+  }
+  return q;
+}
+
+// Narrows a quad to 32 bits, leaves the lane's own running sums in x[0..3] and records in `bad`
+// whether a wanted element lies outside [0, 2^26).
+__device__ __forceinline__ void narrow_quad(const Quad &q, int e, int N, u32 (&x)[4], u32 &bad) {
+  const u32 hi_or = (u32)((u64)q.v[0] >> 32) | (u32)((u64)q.v[1] >> 32) | (u32)((u64)q.v[2] >> 32) |
+                    (u32)((u64)q.v[3] >> 32);
+  const u32 lo_or = (u32)q.v[0] | (u32)q.v[1] | (u32)q.v[2] | (u32)q.v[3];
+  if (hi_or | (lo_or >> 26)) {  // rare: look again, this time only at the elements of this slice
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if ((u32)(e + j) < (u32)N) bad |= (u32)((u64)q.v[j] >> 32) | ((u32)q.v[j] >> 26);
+  }
+  x[0] = (u32)q.v[0];
+  x[1] = x[0] + (u32)q.v[1];
+  x[2] = x[1] + (u32)q.v[2];
+  x[3] = x[2] + (u32)q.v[3];
+}
+
+// True if every 16-byte pair that load_quad_inside would read for this slice is inside the array.
+__device__ __forceinline__ bool slice_is_inside(i64 first, int N, int par, i64 total) {
+  return (par == 0 || first >= 1) && ((((N + par) & 1) == 0) || first + N < total);
+}
+
+template <int SLOTS>
+struct FastLayout {
+  static constexpr int MAXN = 32 * SLOTS;
+  // a prefix array takes slices of up to CAP-1 elements and is written 128 words at a time
+  static constexpr int CAP = (6 * MAXN + 127) / 128 * 128;
+  static constexpr int kInfo = 0;  // uint4 per rank: deadline, base, core, position | GPU flag
+  static constexpr int kQ0 = 4 * MAXN + 4;
+  static constexpr int kQ1 = kQ0 + CAP + 4;
+  static constexpr int kFastWords = kQ1 + CAP;
+  static constexpr int kExactWords = (17 * MAXN + 3) / 4 * 4;  // the exact path: 66 B per task
+  static constexpr int kWords = kFastWords > kExactWords ? kFastWords : kExactWords;
+  static_assert(kWords % 4 == 0 && CAP % 128 == 0 && 4 * MAXN <= CAP, "16-byte aligned rows");
+};
+
+// One 128*NB-element step of the running sums of up to two arrays that share their offsets.
+template <int NB, bool TWO>
+__device__ __forceinline__ void prefix_step(const i64 *__restrict__ X0, const i64 *__restrict__ X1,
+                                            int e0, int N, int par0, int par1, bool inside,
+                                            const i64 *lo0, const i64 *hi0, const i64 *lo1,
+                                            const i64 *hi1, u32 *Q0, u32 *Q1, u32 &carry0,
+                                            u32 &carry1, u32 &bad, int lane) {
+  Quad q0[NB], q1[NB];
+  u32 x0[NB][4], x1[NB][4], i0[NB], i1[NB];
+  if (inside) {
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      load_quad_inside(X0, e0 + 128 * b + 4 * lane - par0, N, q0[b]);
+      if (TWO) load_quad_inside(X1, e0 + 128 * b + 4 * lane - par1, N, q1[b]);
+    }
+  } else {
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      q0[b] = load_quad_edge(X0, e0 + 128 * b + 4 * lane - par0, N, lo0, hi0);
+      if (TWO) q1[b] = load_quad_edge(X1, e0 + 128 * b + 4 * lane - par1, N, lo1, hi1);
+    }
+  }
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    narrow_quad(q0[b], e0 + 128 * b + 4 * lane - par0, N, x0[b], bad);
+    i0[b] = x0[b][3];
+    if (TWO) {
+      narrow_quad(q1[b], e0 + 128 * b + 4 * lane - par1, N, x1[b], bad);
+      i1[b] = x1[b][3];
+    }
+  }
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {  // the warp scans of all blocks side by side
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      const u32 y0 = __shfl_up_sync(kFull, i0[b], d);
+      if (lane >= d) i0[b] += y0;
+      if (TWO) {
+        const u32 y1 = __shfl_up_sync(kFull, i1[b], d);
+        if (lane >= d) i1[b] += y1;
+      }
+    }
+  }
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    if (e0 + 128 * b < N + 1) {
+      const u32 b0 = i0[b] - x0[b][3] + carry0;
+      *reinterpret_cast<uint4 *>(Q0 + e0 + 128 * b + 4 * lane) =
+          make_uint4(x0[b][0] + b0, x0[b][1] + b0, x0[b][2] + b0, x0[b][3] + b0);
+      carry0 += __shfl_sync(kFull, i0[b], 31);
+      if (TWO) {
+        const u32 b1 = i1[b] - x1[b][3] + carry1;
+        *reinterpret_cast<uint4 *>(Q1 + e0 + 128 * b + 4 * lane) =
+            make_uint4(x1[b][0] + b1, x1[b][1] + b1, x1[b][2] + b1, x1[b][3] + b1);
+        carry1 += __shfl_sync(kFull, i1[b], 31);
+      }
+    }
   }
 }
 
 // MODE: 0 GCAPS self-suspension, 1 GCAPS busy-waiting, 2 RR self-suspension, 3 RR busy-waiting.
 // Returns false, having written nothing, if the taskset is not eligible for 32-bit arithmetic
 // (or is invalid): the caller then runs the exact 64-bit path, which also does the validation.
+//
+// Until the per-task sums are known lane l holds the tasks at positions l, l+32, ... ("slots").
+// Then every task's values move through shared memory to the lane that owns its rank, so that the
+// interferers of the task of rank `pos` sit in lanes (pos-1) % 32 downwards of slots up to
+// (pos-1) / 32 and higher slots can be skipped.
 template <int SLOTS, int MODE>
 __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane) {
-  constexpr int MAXN = 32 * SLOTS;
-  constexpr int CAP = 10 * MAXN;  // elements one prefix buffer can take
+  typedef FastLayout<SLOTS> Lay;
+  constexpr int MAXN = Lay::MAXN, CAP = Lay::CAP;
+  constexpr int BC = SLOTS <= 4 ? SLOTS : 4;  // 128-element steps whose loads are issued together
+  constexpr int BG = SLOTS <= 2 ? SLOTS : 2;
   constexpr bool kGcaps = MODE < 2;
   const bool literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
-  u32 *P0 = buf, *P1 = buf + CAP + 32;
+  uint4 *info = reinterpret_cast<uint4 *>(buf + Lay::kInfo);
+  u32 *Q0 = buf + Lay::kQ0, *Q1 = buf + Lay::kQ1;
 
-  // ---- stage: per-task scalars, lane = position -------------------------------------------
-  const i64 cfirst = p.cseg_off[a] - p.cseg_base, gfirst = p.gseg_off[a] - p.gseg_base;
-  const i64 Nc64 = p.cseg_off[a + n] - p.cseg_base - cfirst;
-  const i64 Ng64 = p.gseg_off[a + n] - p.gseg_base - gfirst;
-  if (cfirst < 0 || Nc64 < 0 || cfirst + Nc64 > p.n_csegs || Nc64 > CAP || gfirst < 0 || Ng64 < 0 ||
-      gfirst + Ng64 > p.n_gsegs || Ng64 > CAP)
-    return false;
-  const int Nc = (int)Nc64, Ng = (int)Ng64;
+  // ---- stage: per-task scalars, lane = position; rank ----------------------------------------
   u32 T[SLOTS], D[SLOTS], core[SLOTS];
-  int prio[SLOTS], c0[SLOTS], g0[SLOTS];
-  bool ok = true, prio_small = true;
+  int rank[SLOTS], c0[SLOTS], g0[SLOTS];
+  bool ok = true;
+  int Nc, Ng;
+  i64 cfirst, gfirst;
+  {
+    i64 t64[SLOTS], d64[SLOTS], pr[SLOTS], c64[SLOTS], co[SLOTS], go[SLOTS];
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) {
-    const int i = lane + 32 * s;
-    const bool v = i < n;
-    const i64 k = a + (v ? i : 0);
-    const i64 t64 = p.period[k], d64 = p.deadline[k], pr = p.priority[k], c64 = p.core[k];
-    const i64 co = p.cseg_off[k] - p.cseg_base - cfirst, go = p.gseg_off[k] - p.gseg_base - gfirst;
-    ok &= !v || ((u64)(t64 - 2) < (u64)(kFastLimit - 2) && d64 >= 1 && d64 <= t64 &&
-                 (u64)c64 <= (u64)GCAPS_RTA_MAX_CORE && (u64)co <= (u64)Nc && (u64)go <= (u64)Ng);
-    prio_small &= !v || pr == (i64)(int)pr;
-    T[s] = v ? (u32)t64 : 2u;
-    D[s] = (u32)d64;
-    core[s] = (u32)c64;
-    prio[s] = v ? (int)pr : (int)0x80000000;
-    c0[s] = v ? (int)co : Nc;
-    g0[s] = v ? (int)go : Ng;
+    for (int s = 0; s < SLOTS; ++s) {  // all loads of the taskset's per-task arrays in flight
+      const i64 k = a + (lane + 32 * s < n ? lane + 32 * s : 0);
+      t64[s] = p.period[k], d64[s] = p.deadline[k], pr[s] = p.priority[k], c64[s] = p.core[k];
+      co[s] = p.cseg_off[k], go[s] = p.gseg_off[k];
+    }
+    const i64 cend = p.cseg_off[a + n] - p.cseg_base, gend = p.gseg_off[a + n] - p.gseg_base;
+    cfirst = __shfl_sync(kFull, co[0], 0) - p.cseg_base;
+    gfirst = __shfl_sync(kFull, go[0], 0) - p.gseg_base;
+    const i64 Nc64 = cend - cfirst, Ng64 = gend - gfirst;
+    if (cfirst < 0 || Nc64 < 0 || cend > p.n_csegs || Nc64 >= CAP || gfirst < 0 || Ng64 < 0 ||
+        gend > p.n_gsegs || Ng64 >= CAP)
+      return false;
+    Nc = (int)Nc64, Ng = (int)Ng64;
+    u32 high = 0;  // any set bit: some value does not fit the 32-bit path
+    int prio[SLOTS];
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const bool v = lane + 32 * s < n;
+      const i64 rc = co[s] - p.cseg_base - cfirst, rg = go[s] - p.gseg_base - gfirst;
+      const u32 h = (u32)((u64)t64[s] >> 32) | (u32)((u64)d64[s] >> 32) | (u32)((u64)c64[s] >> 32) |
+                    (u32)((u64)rc >> 32) | (u32)((u64)rg >> 32) |
+                    (u32)(((u64)pr[s] + 0x80000000ull) >> 32);
+      T[s] = v ? (u32)t64[s] : 2u;
+      D[s] = (u32)d64[s];
+      core[s] = (u32)c64[s];
+      prio[s] = v ? (int)pr[s] : (int)0x80000000;
+      c0[s] = v ? (int)rc : Nc;
+      g0[s] = v ? (int)rg : Ng;
+      high |= v ? h : 0u;
+      // 2 <= T < 2^26, 1 <= D <= T, core < 2^31, offsets inside the slice
+      ok &= T[s] - 2u < kFastLimit - 2u && (!v || (D[s] - 1u < T[s] && (int)core[s] >= 0)) &&
+            (u32)c0[s] <= (u32)Nc && (u32)g0[s] <= (u32)Ng;
+    }
+    if (__any_sync(kFull, high != 0 || !ok)) return false;  // (a wide priority also lands here)
+    // order: rank by (priority desc, position asc)
+    int m = prio[0];
+#pragma unroll
+    for (int s = 1; s < SLOTS; ++s) m = prio[s] > m ? prio[s] : m;
+    const int pmax = __reduce_max_sync(kFull, m);
+    bool dense = true;  // distinct priorities max-n+1 .. max: the rank is max - priority
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const u32 r = (u32)pmax - (u32)prio[s];
+      const bool v = lane + 32 * s < n;
+      dense &= !v || r < (u32)n;
+      rank[s] = v ? (int)r : MAXN;
+    }
+    dense = __all_sync(kFull, dense);
+    if (dense) {
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s)
+        if (lane + 32 * s < n) Q0[rank[s]] = (u32)(lane + 32 * s);
+      __syncwarp();
+      bool uniq = true;
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s)
+        if (lane + 32 * s < n) uniq &= Q0[rank[s]] == (u32)(lane + 32 * s);
+      dense = __all_sync(kFull, uniq);
+      __syncwarp();
+    }
+    if (!dense) {  // any priorities: count the tasks that come before
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s) {
+        const int i = lane + 32 * s;
+        int r = 0;
+        for (int q = 0; q < n; ++q) {
+          const int pq = (int)p.priority[a + q];
+          r += (pq > prio[s] || (pq == prio[s] && q < i)) ? 1 : 0;
+        }
+        rank[s] = i < n ? r : MAXN;
+      }
+    }
   }
   // end offsets: the next task's start (positions beyond n hold the total)
   int c1[SLOTS], g1[SLOTS];
@@ -486,57 +662,87 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   }
   if (!__all_sync(kFull, ok)) return false;
 
-  // ---- aggregate: prefix sums of the segment arrays, per-task sums as differences ---------
+  // ---- aggregate: running sums of the segment arrays; per-task sums are differences --------
   u32 A[SLOTS], Ge[SLOTS], S[SLOTS];  // C+G^m, G^e, and 2*eps*eta (GCAPS) or (L+theta)*slices (RR)
-  scan_one(p.cseg_wcet + cfirst, Nc, P0, lane, ok);
+  u32 bad = 0;
+  const i64 *__restrict__ Xc = p.cseg_wcet + cfirst;
+  const i64 *__restrict__ Xm = p.gseg_misc + gfirst, *__restrict__ Xe = p.gseg_exec + gfirst;
+  const int parc = (int)(((uintptr_t)Xc >> 3) & 1), parm = (int)(((uintptr_t)Xm >> 3) & 1);
+  const int pare = (int)(((uintptr_t)Xe >> 3) & 1);
+  if (lane == 0) Q0[-1] = 0, Q1[-1] = 0;
+  {  // CPU segments -> Q0
+    const bool inside = slice_is_inside(cfirst, Nc, parc, p.n_csegs);
+    u32 carry = 0, unused = 0;
+    for (int e0 = 0; e0 < Nc + parc; e0 += 128 * BC)
+      prefix_step<BC, false>(Xc, Xc, e0, Nc, parc, parc, inside, p.cseg_wcet, p.cseg_wcet + p.n_csegs,
+                             p.cseg_wcet, p.cseg_wcet, Q0, Q0, carry, unused, bad, lane);
+  }
   __syncwarp();
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) A[s] = P0[c1[s]] - P0[c0[s]];
+  for (int s = 0; s < SLOTS; ++s) A[s] = Q0[c1[s] - 1 + parc] - Q0[c0[s] - 1 + parc];
   __syncwarp();
-  {  // G^m into P0 and G^e into P1, interleaved
-    const i64 *__restrict__ Xm = p.gseg_misc + gfirst, *__restrict__ Xe = p.gseg_exec + gfirst;
+  {  // G^m -> Q0, G^e -> Q1
+    const bool inside = slice_is_inside(gfirst, Ng, parm, p.n_gsegs) &&
+                        slice_is_inside(gfirst, Ng, pare, p.n_gsegs);
     u32 cm = 0, ce = 0;
-    if (lane == 0) P0[0] = 0, P1[0] = 0;
-    for (int e0 = 0; e0 < Ng; e0 += 32) {
-      const int e = e0 + lane;
-      const i64 vm = e < Ng ? Xm[e] : 0, ve = e < Ng ? Xe[e] : 0;
-      ok &= (u64)vm < kFastLimit && (u64)ve < kFastLimit;
-      u32 xm = (u32)vm, xe = (u32)ve;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const u32 ym = __shfl_up_sync(kFull, xm, d), ye = __shfl_up_sync(kFull, xe, d);
-        if (lane >= d) xm += ym, xe += ye;
-      }
-      xm += cm, xe += ce;
-      if (e < Ng) P0[e + 1] = xm, P1[e + 1] = xe;
-      cm = __shfl_sync(kFull, xm, 31), ce = __shfl_sync(kFull, xe, 31);
-    }
+    for (int e0 = 0; e0 < Ng + 1; e0 += 128 * BG)
+      prefix_step<BG, true>(Xm, Xe, e0, Ng, parm, pare, inside, p.gseg_misc, p.gseg_misc + p.n_gsegs,
+                            p.gseg_exec, p.gseg_exec + p.n_gsegs, Q0, Q1, cm, ce, bad, lane);
   }
   __syncwarp();
   u32 eta[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    const u32 C = A[s], Gm = P0[g1[s]] - P0[g0[s]];
-    Ge[s] = P1[g1[s]] - P1[g0[s]];
+    const u32 Gm = Q0[g1[s] - 1 + parm] - Q0[g0[s] - 1 + parm];
+    Ge[s] = Q1[g1[s] - 1 + pare] - Q1[g0[s] - 1 + pare];
     eta[s] = (u32)(g1[s] - g0[s]);
-    A[s] = C + Gm;
-    ok &= C < kFastLimit && Gm < kFastLimit && Ge[s] < kFastLimit && A[s] < kFastLimit;
+    bad |= (A[s] | Gm | Ge[s]) >> 26;
+    A[s] += Gm;
+    bad |= A[s] >> 26;
   }
   __syncwarp();
-  if (!kGcaps) {  // Eq. 3: slices of every pure GPU part, summed per task
-    const i64 *__restrict__ Xe = p.gseg_exec + gfirst;
+  if (!kGcaps) {  // Eq. 3: slices of every pure GPU part, summed per task (values already checked)
+    const bool inside = slice_is_inside(gfirst, Ng, pare, p.n_gsegs);
     u32 carry = 0;
-    if (lane == 0) P0[0] = 0;
-    for (int e0 = 0; e0 < Ng; e0 += 32) {
-      const int e = e0 + lane;
-      const u32 ve = e < Ng ? (u32)Xe[e] : 0u;  // range was checked by the pass above
-      u32 sl;
-      if (p.l_mode == 0) sl = __umulhi(ve + (u32)p.L - 1u, p.l_magic) >> p.l_shift;
-      else if (p.l_mode == 1) sl = ve;
-      else sl = ve > 0 ? 1u : 0u;
-      const u32 x = warp_incl_scan(sl, lane) + carry;
-      if (e < Ng) P0[e + 1] = x;
-      carry = __shfl_sync(kFull, x, 31);
+    for (int e0 = 0; e0 < Ng + 1; e0 += 128 * BG) {
+      Quad qe[BG];
+      u32 x[BG][4], incl[BG];
+#pragma unroll
+      for (int b = 0; b < BG; ++b) {
+        if (inside) load_quad_inside(Xe, e0 + 128 * b + 4 * lane - pare, Ng, qe[b]);
+        else qe[b] = load_quad_edge(Xe, e0 + 128 * b + 4 * lane - pare, Ng, p.gseg_exec, p.gseg_exec + p.n_gsegs);
+      }
+#pragma unroll
+      for (int b = 0; b < BG; ++b) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          // a neighbour's element may be large: keep it below 2^26 so the division stays exact
+          const u32 w = (u32)qe[b].v[j] & (kFastLimit - 1);
+          u32 sl;
+          if (p.l_mode == 0) sl = __umulhi(w + (u32)p.L - 1u, p.l_magic) >> p.l_shift;
+          else if (p.l_mode == 1) sl = w;
+          else sl = w > 0 ? 1u : 0u;
+          x[b][j] = sl + (j > 0 ? x[b][j - 1] : 0u);
+        }
+        incl[b] = x[b][3];
+      }
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+#pragma unroll
+        for (int b = 0; b < BG; ++b) {
+          const u32 y = __shfl_up_sync(kFull, incl[b], d);
+          if (lane >= d) incl[b] += y;
+        }
+      }
+#pragma unroll
+      for (int b = 0; b < BG; ++b) {
+        if (e0 + 128 * b < Ng + 1) {
+          const u32 before = incl[b] - x[b][3] + carry;
+          *reinterpret_cast<uint4 *>(Q0 + e0 + 128 * b + 4 * lane) =
+              make_uint4(x[b][0] + before, x[b][1] + before, x[b][2] + before, x[b][3] + before);
+          carry += __shfl_sync(kFull, incl[b], 31);
+        }
+      }
     }
     __syncwarp();
   }
@@ -544,181 +750,136 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   int n_gpu = 0;  // N_g
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(kFull, eta[s] > 0));
+  const u32 ovh = (u32)p.ovh;  // the fast path is only entered with eps, theta < 2^20
   u32 base[SLOTS];
-  const u64 ovh = (u64)p.ovh;
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    u64 b64;
     if (kGcaps) {
-      const u64 star = 2 * ovh * eta[s];  // eta < 64, ovh <= 2^40
-      ok &= star < kFastLimit;
-      S[s] = (u32)star;
-      b64 = (u64)A[s] + Ge[s] + star + ((u64)eta[s] + 1) * ovh;  // C_i + G*_i + B^C_i
+      S[s] = 2 * ovh * eta[s];                                 // eta < 64: below 2^27
+      base[s] = A[s] + Ge[s] + S[s] + (eta[s] + 1) * ovh;        // C_i + G*_i + B^C_i, below 2^29
+      bad |= S[s] >> 26;
     } else {
-      const u64 slices = P0[g1[s]] - P0[g0[s]];
+      const u64 slices = Q0[g1[s] - 1 + pare] - Q0[g0[s] - 1 + pare];
       const u64 lt = (u64)p.L + ovh;  // <= 2^41
       u64 B = slices == 0 ? 0 : (lt >= kFastClamp ? kFastClamp : lt * slices);  // < 2^26 * 2^32
       if (B > kFastClamp) B = kFastClamp;
       S[s] = (u32)B;
-      u64 ie = eta[s] > 0 ? B * (u64)(n_gpu - 1) : 0;  // Lemma 1
-      b64 = (u64)A[s] + Ge[s] + ie;
+      const u64 b64 = (u64)A[s] + Ge[s] + (eta[s] > 0 ? B * (u64)(n_gpu - 1) : 0);  // Lemma 1
+      base[s] = b64 > (u64)(2 * kFastClamp) ? 2 * kFastClamp : (u32)b64;
     }
-    base[s] = b64 > (u64)(2 * kFastClamp) ? 2 * kFastClamp : (u32)b64;
+    base[s] = base[s] > 2 * kFastClamp ? 2 * kFastClamp : base[s];
   }
-  if (!__all_sync(kFull, ok)) return false;
+  if (__any_sync(kFull, bad != 0)) return false;
   __syncwarp();
-
-  // ---- order ---------------------------------------------------------------------------------
-  int rank[SLOTS];
-  bool dense = __all_sync(kFull, prio_small);
-  if (dense) {  // distinct priorities max-n+1 .. max: the rank is max - priority
-    int m = prio[0];
-#pragma unroll
-    for (int s = 1; s < SLOTS; ++s) m = prio[s] > m ? prio[s] : m;
-    const int pmax = __reduce_max_sync(kFull, m);
-    bool in = true;
-#pragma unroll
-    for (int s = 0; s < SLOTS; ++s) {
-      const i64 r = (i64)pmax - (i64)prio[s];
-      const bool v = lane + 32 * s < n;
-      in &= !v || r < (i64)n;
-      rank[s] = v ? (int)r : 0;
-    }
-    dense = __all_sync(kFull, in);
-    if (dense) {
-#pragma unroll
-      for (int s = 0; s < SLOTS; ++s)
-        if (lane + 32 * s < n) buf[rank[s]] = (u32)(lane + 32 * s);
-      __syncwarp();
-      bool uniq = true;
-#pragma unroll
-      for (int s = 0; s < SLOTS; ++s)
-        if (lane + 32 * s < n) uniq &= buf[rank[s]] == (u32)(lane + 32 * s);
-      dense = __all_sync(kFull, uniq);
-      __syncwarp();
-    }
-  }
-  if (!dense) {  // any priorities: count the tasks that come before
-#pragma unroll
-    for (int s = 0; s < SLOTS; ++s) {
-      const int i = lane + 32 * s;
-      const i64 pi = p.priority[a + (i < n ? i : 0)];
-      int r = 0;
-      for (int q = 0; q < n; ++q) {
-        const i64 pq = p.priority[a + q];
-        r += (pq > pi || (pq == pi && q < i)) ? 1 : 0;
-      }
-      rank[s] = r;
-    }
-  }
-  // ---- move the per-task values to the lane that owns the rank -----------------------------
-  // word w of rank r sits at buf[w * MAXN + r]; words 1, 2, 6, 7 are read again per task below
+  // ---- move every task to the lane that owns its rank -------------------------------------
+  uint4 *xch = reinterpret_cast<uint4 *>(Q0);  // by rank: T, C+G^m, G^e, S  (Q0, Q1 are dead now)
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    const int i = lane + 32 * s;
-    if (i < n) {
-      const int r = rank[s];
-      buf[0 * MAXN + r] = T[s];
-      buf[1 * MAXN + r] = D[s];
-      buf[2 * MAXN + r] = base[s];
-      buf[3 * MAXN + r] = A[s];
-      buf[4 * MAXN + r] = Ge[s];
-      buf[5 * MAXN + r] = S[s];
-      buf[6 * MAXN + r] = core[s];
-      buf[7 * MAXN + r] = (u32)i | (eta[s] > 0 ? 0x10000u : 0u);
+    if (lane + 32 * s < n) {
+      info[rank[s]] = make_uint4(D[s], base[s], core[s], (u32)(lane + 32 * s) | (eta[s] > 0 ? 0x10000u : 0u));
+      xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], S[s]);
     }
   }
   __syncwarp();
-  u32 magic[SLOTS], shift[SLOTS], Tm1[SLOTS], pos_of[SLOTS];
+  u32 Tm1[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS];
   bool gpu[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + 32 * s;
-    const bool v = r < n;
-    const u32 Tr = v ? buf[0 * MAXN + r] : 2u;
-    A[s] = v ? buf[3 * MAXN + r] : 0u;
-    Ge[s] = v ? buf[4 * MAXN + r] : 0u;
-    S[s] = v ? buf[5 * MAXN + r] : 0u;
-    core[s] = v ? buf[6 * MAXN + r] : 0xffffffffu;
-    const u32 meta = v ? buf[7 * MAXN + r] : 0u;
-    pos_of[s] = meta & 0xffffu;
-    gpu[s] = (meta & 0x10000u) != 0;
-    Tm1[s] = Tr - 1;
-    make_reciprocal(Tr, magic[s], shift[s]);
+    const uint4 x = r < n ? xch[r] : make_uint4(2u, 0u, 0u, 0u);
+    const uint4 f = r < n ? info[r] : make_uint4(0u, 0u, 0xffffffffu, 0u);
+    Tm1[s] = x.x - 1, A[s] = x.y, Ge[s] = x.z, S[s] = x.w;
+    core[s] = f.z, pos_of[s] = f.w & 0xffffu, gpu[s] = (f.w & 0x10000u) != 0;
+    if (MODE == 0) {
+      Wa[s] = A[s] + (gpu[s] ? S[s] : 0u);  // Lemma 15: C_h, or C_h + G^{m*}_h
+      Wb[s] = gpu[s] ? Ge[s] + S[s] : 0u;   // Lemma 13, other cores: G^{e*}_h
+    } else if (MODE == 1) {
+      Wa[s] = A[s];                         // Lemma 12
+      Wb[s] = gpu[s] ? Ge[s] + S[s] : 0u;   // Lemmas 10, 11: G^{e*}_h
+    } else {
+      Wa[s] = A[s];                         // Lemmas 5, 7
+      Wb[s] = gpu[s] ? S[s] : 0u;           // Lemma 4: (L+theta) * slices
+    }
   }
 
   // ---- iterate in rank order ------------------------------------------------------------------
+  u32 magic[SLOTS], shift[SLOTS];         // reciprocal of T_h, made when the slot is first needed
   u32 Jc[SLOTS], Jg[SLOTS], Rown[SLOTS];  // jitters with T_h - 1 folded in (ceiling), own result
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Rown[s] = 0;
+  for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Tm1[s], Rown[s] = 0, magic[s] = 0, shift[s] = 0;
   int n_done = n;
-  i64 verdict = 0;
+  int verdict = 0;
   for (int pos = 0; pos < n; ++pos) {
-    const u32 Di = buf[1 * MAXN + pos], base_i = buf[2 * MAXN + pos], core_i = buf[6 * MAXN + pos];
-    const bool gi = (buf[7 * MAXN + pos] & 0x10000u) != 0;
+    const uint4 f = info[pos];
+    const u32 Di = f.x, base_i = f.y, core_i = f.z;
+    const bool gi = (f.w & 0x10000u) != 0;
+    const int smax = (pos - 1) >> 5;  // -1 for the first task: nothing interferes
+    if ((pos & 31) == 1) {            // the first task that looks at slot smax
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s)
+        if (s == smax) make_reciprocal(Tm1[s] + 1, magic[s], shift[s]);
+    }
     u32 nu = 0;
     if (MODE == 3) {  // Lemma 4: N_g - |{h in hpp(i): GPU-using}| + 1
       int c = 0;
 #pragma unroll
       for (int s = 0; s < SLOTS; ++s)
-        c += __popc(__ballot_sync(kFull, lane + 32 * s < pos && core[s] == core_i && gpu[s]));
+        if (s <= smax) c += __popc(__ballot_sync(kFull, lane + 32 * s < pos && core[s] == core_i && gpu[s]));
       nu = (u32)(n_gpu - c + 1);
     }
     // the (J, W) pairs of this task's interferers; W = 0 where a pair does not apply
-    u32 J1[SLOTS], W1[SLOTS], J2[SLOTS], W2[SLOTS];
+    u32 J1[SLOTS], W1[SLOTS], W2[SLOTS];
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
-      const bool act = lane + 32 * s < pos;
-      const bool same = core[s] == core_i, gh = gpu[s];
-      u32 w1 = 0, w2 = 0, j1 = Tm1[s], j2 = Tm1[s];
-      if (MODE == 0) {
-        if (same) {  // Lemma 15
-          w1 = A[s] + (gh ? S[s] : 0u);
-          j1 = gh ? Jc[s] : Tm1[s];
-          if (gh && gi) w2 = Ge[s], j2 = Jg[s];  // Lemma 13, same core
-        } else if (gh && gi) {
-          w1 = Ge[s] + S[s], j1 = Jg[s];  // Lemma 13, other cores
+      J1[s] = 0, W1[s] = 0, W2[s] = 0;
+      if (s <= smax) {
+        const bool act = lane + 32 * s < pos;
+        const bool same = core[s] == core_i;
+        u32 w1, w2 = 0, j1;
+        if (MODE == 0) {
+          w1 = same ? Wa[s] : (gi ? Wb[s] : 0u);           // Lemma 15 / Lemma 13 (other cores)
+          j1 = same ? Jc[s] : Jg[s];
+          w2 = (same && gi && gpu[s]) ? Ge[s] : 0u;        // Lemma 13 (same core), jitter J^g
+        } else if (MODE == 1) {
+          w1 = same ? Wa[s] + ((gi || !literal) ? Wb[s] : 0u) : Wb[s];  // Lemmas 12+10 / 10, 11
+          j1 = same ? Tm1[s] : Jg[s];
+        } else if (MODE == 2) {
+          w1 = same ? Wa[s] : 0u;                          // Lemma 7
+          j1 = Jc[s];
+        } else {
+          const u64 w = (u64)Wa[s] + (u64)Wb[s] * nu;      // Lemmas 5 and 4
+          w1 = same ? (w > kFastClamp ? kFastClamp : (u32)w) : 0u;
+          j1 = Tm1[s];
         }
-      } else if (MODE == 1) {
-        if (same) {
-          w1 = A[s] + ((gh && (gi || !literal)) ? Ge[s] + S[s] : 0u);  // Lemmas 12, 10
-        } else if (gh) {
-          w1 = Ge[s] + S[s], j1 = Jg[s];  // Lemma 10 / Lemma 11
-        }
-      } else if (MODE == 2) {
-        if (same) w1 = A[s], j1 = (gh || literal) ? Jc[s] : Tm1[s];  // Lemma 7
-      } else {
-        if (same) {  // Lemmas 5 and 4
-          const u64 w = (u64)A[s] + (gh ? (u64)S[s] * nu : 0ull);
-          w1 = w > kFastClamp ? kFastClamp : (u32)w;
-        }
+        J1[s] = j1, W1[s] = act ? w1 : 0u, W2[s] = act ? w2 : 0u;
       }
-      J1[s] = j1, W1[s] = act ? w1 : 0u, J2[s] = j2, W2[s] = act ? w2 : 0u;
     }
-    const int smax = pos == 0 ? -1 : (pos - 1) >> 5;
     u32 R = base_i;
-    i64 v = 0;
-    i64 sweeps = 0;
+    int v = 0;
+    int sweeps = 0;
     for (;;) {
       if (R > Di) {
         v = GCAPS_WCRT_MISS;
         break;
       }
-      if (sweeps >= GCAPS_RTA_ITER_CAP) {
+      if (sweeps >= (int)GCAPS_RTA_ITER_CAP) {
         v = GCAPS_WCRT_ITER_LIMIT;
         break;
       }
       sweeps += 1;
-      u64 acc = 0;
+      u32 next = base_i;
+      if (smax >= 0) {
+        u64 acc = 0;
 #pragma unroll
-      for (int s = 0; s < SLOTS; ++s) {
-        if (s <= smax) {
-          acc += (u64)(__umulhi(R + J1[s], magic[s]) >> shift[s]) * W1[s];
-          if (MODE == 0) acc += (u64)(__umulhi(R + J2[s], magic[s]) >> shift[s]) * W2[s];
+        for (int s = 0; s < SLOTS; ++s) {
+          if (s <= smax) {
+            acc += (u64)(__umulhi(R + J1[s], magic[s]) >> shift[s]) * W1[s];
+            if (MODE == 0) acc += (u64)(__umulhi(R + Jg[s], magic[s]) >> shift[s]) * W2[s];
+          }
         }
+        const u32 part = acc > (u64)kFastClamp ? kFastClamp : (u32)acc;
+        next += __reduce_add_sync(kFull, part);
       }
-      const u32 part = acc > (u64)kFastClamp ? kFastClamp : (u32)acc;
-      const u32 next = base_i + __reduce_add_sync(kFull, part);
       if (next == R) break;
       R = next;
     }
@@ -727,12 +888,13 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       verdict = v;
       break;
     }
-    // publish: the owner of this rank keeps R_i and its jitters J^c = R - (C+G^m), J^g = R - G^e
+    // publish: the owner keeps R_i and its jitters J^c = R - (C+G^m), J^g = R - G^e (a CPU-only
+    // task has no J^c unless the printed form of Lemma 7 is asked for)
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
       if (lane + 32 * s == pos) {
         Rown[s] = R;
-        Jc[s] = R - A[s] + Tm1[s];
+        if (MODE == 0 ? gpu[s] : (MODE == 2 ? (gpu[s] || literal) : false)) Jc[s] = R - A[s] + Tm1[s];
         Jg[s] = R - Ge[s] + Tm1[s];
       }
     }
@@ -742,44 +904,109 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + 32 * s;
     if (r < n)
-      p.out_wcrt[a + pos_of[s]] = r < n_done ? (i64)Rown[s] : (r == n_done ? verdict : (i64)GCAPS_WCRT_SKIPPED);
+      p.out_wcrt[a + pos_of[s]] =
+          r < n_done ? (i64)Rown[s] : (r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED);
   }
   if (lane == 0) p.out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
   __syncwarp();
   return true;
 }
 
-// shared memory of one warp, in 32-bit words: two prefix buffers of 10*MAXN+32 words each; the
-// image of the exact path (GroupSmem, 74 bytes per task) fits in the same space
-template <int SLOTS>
-__host__ __device__ constexpr int warp_words() { return 20 * 32 * SLOTS + 64; }
+__device__ __forceinline__ void prefetch_l2(const void *ptr) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
+
+// What a warp knows in advance about one taskset of its chunk.
+struct Ahead {
+  i64 t, a;        // taskset index, first task
+  i64 c_lo, g_lo;  // first CPU segment, first GPU segment
+  int n, nc, ng;   // tasks, CPU segments, GPU segments; nc = ng = 0 unless safe to prefetch
+  int pf;          // 1 if the task range is one the fast path could take
+};
 
 // Persistent launch over one size bin: warps pull chunks of tasksets from the bin's counter.
+// While one taskset is analysed the input of the next one is already on its way into L2.
 template <int SLOTS, int MODE>
 __global__ void __launch_bounds__(kBlockThreads) rta_kernel(KParams p, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  typedef FastLayout<SLOTS> Lay;
   constexpr int MAXN = 32 * SLOTS;
   constexpr int kChunk = 4;  // tasksets per pull
-  static_assert(sizeof(GroupSmem<MAXN>) <= sizeof(u32) * warp_words<SLOTS>(), "exact path fits");
+  static_assert(sizeof(GroupSmem<MAXN>) <= sizeof(u32) * Lay::kWords, "exact path fits");
+  static_assert(6 * MAXN <= Lay::CAP, "prefetched ranges are ranges the fast path accepts");
   const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * warp_words<SLOTS>();
+  u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * Lay::kWords;
   const unsigned int start = p.hdr->bin_start[bin], count = p.hdr->bin_count[bin];
-  for (;;) {
-    unsigned int first = 0;
-    if (lane == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
-    first = __shfl_sync(kFull, first, 0);
-    if (first >= count) break;
-    const unsigned int last = first + kChunk < count ? first + kChunk : count;
-    for (unsigned int idx = first; idx < last; ++idx) {
-      const i64 t = (i64)p.perm[start + idx];
-      const i64 a = p.task_off[t] - p.task_base, b = p.task_off[t + 1] - p.task_base;
+  const bool fast_call = p.ovh < (1 << 20);  // keeps 2*eps*eta and (eta+1)*eps in 32 bits
+
+  // lanes 0..kChunk-1 each look up one taskset of a chunk
+  auto look_up = [&](unsigned int first, Ahead &me) {
+    me.t = 0, me.a = 0, me.c_lo = me.g_lo = 0, me.n = me.nc = me.ng = 0, me.pf = 0;
+    if (lane < kChunk && first < count && first + lane < count) {
+      me.t = (i64)p.perm[start + first + lane];
+      me.a = p.task_off[me.t] - p.task_base;
+      const i64 b = p.task_off[me.t + 1] - p.task_base;
+      if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN) {
+        me.pf = 1, me.n = (int)(b - me.a);
+        me.c_lo = p.cseg_off[me.a] - p.cseg_base, me.g_lo = p.gseg_off[me.a] - p.gseg_base;
+        const i64 c_hi = p.cseg_off[b] - p.cseg_base, g_hi = p.gseg_off[b] - p.gseg_base;
+        if (me.c_lo >= 0 && c_hi <= p.n_csegs && c_hi - me.c_lo <= 6 * MAXN && c_hi > me.c_lo)
+          me.nc = (int)(c_hi - me.c_lo);
+        if (me.g_lo >= 0 && g_hi <= p.n_gsegs && g_hi - me.g_lo <= 6 * MAXN && g_hi > me.g_lo)
+          me.ng = (int)(g_hi - me.g_lo);
+      }
+    }
+  };
+  // all lanes: pull the lines of taskset c of the chunk towards L2 (16 elements per line; only
+  // addresses inside the arrays are named)
+  auto prefetch = [&](const Ahead &me, int c) {
+    if (__shfl_sync(kFull, me.pf, c) == 0) return;
+    const i64 a = __shfl_sync(kFull, me.a, c);
+    const i64 c_lo = __shfl_sync(kFull, me.c_lo, c), g_lo = __shfl_sync(kFull, me.g_lo, c);
+    const int n = __shfl_sync(kFull, me.n, c), nc = __shfl_sync(kFull, me.nc, c);
+    const int ng = __shfl_sync(kFull, me.ng, c);
+    for (int e = 16 * lane; e < n; e += 16 * 32) {
+      prefetch_l2(p.period + a + e), prefetch_l2(p.deadline + a + e), prefetch_l2(p.priority + a + e);
+      prefetch_l2(p.core + a + e), prefetch_l2(p.cseg_off + a + e), prefetch_l2(p.gseg_off + a + e);
+    }
+    for (int e = 16 * lane; e < nc; e += 16 * 32) prefetch_l2(p.cseg_wcet + c_lo + e);
+    for (int e = 16 * lane; e < ng; e += 16 * 32)
+      prefetch_l2(p.gseg_misc + g_lo + e), prefetch_l2(p.gseg_exec + g_lo + e);
+  };
+
+  unsigned int first = 0;
+  if (lane == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
+  first = __shfl_sync(kFull, first, 0);
+  Ahead cur;
+  look_up(first, cur);
+  if (first < count) prefetch(cur, 0);
+  while (first < count) {
+    unsigned int nfirst = 0;
+    if (lane == 0) nfirst = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
+    Ahead nxt;
+    nxt.t = 0, nxt.a = 0, nxt.c_lo = nxt.g_lo = 0, nxt.n = nxt.nc = nxt.ng = 0, nxt.pf = 0;
+    const int in_chunk = count - first < (unsigned int)kChunk ? (int)(count - first) : kChunk;
+    for (int c = 0; c < in_chunk; ++c) {
+      if (c + 1 < in_chunk) prefetch(cur, c + 1);
+      if (c == 1 || in_chunk == 1) {  // the next chunk's index has arrived by now
+        nfirst = __shfl_sync(kFull, nfirst, 0);
+        look_up(nfirst, nxt);
+      }
+      if (c == in_chunk - 1 && nfirst < count) prefetch(nxt, 0);
+      const i64 t = __shfl_sync(kFull, cur.t, c), a = __shfl_sync(kFull, cur.a, c);
+      const int n = __shfl_sync(kFull, cur.n, c);
       bool done = false;
-      if (a >= 0 && b > a && b <= p.n_tasks && b - a <= MAXN)
-        done = analyse_fast<SLOTS, MODE>(p, t, a, (int)(b - a), buf, lane);
+      if (fast_call && __shfl_sync(kFull, cur.pf, c) != 0)
+        done = analyse_fast<SLOTS, MODE>(p, t, a, n, buf, lane);
       __syncwarp();
-      if (!done) analyse_taskset<32, MAXN>(p, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, kFull);
+      if (!done) {
+        // the exact path reads task_off again and validates everything itself
+        analyse_taskset<32, MAXN>(p, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, kFull);
+      }
       __syncwarp();
     }
+    first = nfirst;
+    cur = nxt;
   }
 }
 
@@ -909,7 +1136,7 @@ void fill_params(KParams *p, const gcaps_tasksets_t *ts, int64_t n_tasksets, int
 template <int SLOTS, int MODE>
 cudaError_t launch_bin(const KParams &p, int bin, int sm_count, cudaStream_t st) {
   constexpr int kWarps = kBlockThreads / 32;
-  const size_t smem = sizeof(u32) * warp_words<SLOTS>() * kWarps;
+  const size_t smem = sizeof(u32) * FastLayout<SLOTS>::kWords * kWarps;
   static int blocks_per_sm[64] = {0};  // per device; 0 = not set up yet
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);

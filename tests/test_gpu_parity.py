@@ -212,6 +212,26 @@ def test_values_around_the_32_bit_path_limit():
             assert_parity(b, policy, L, ovh, "limit L=%d ovh=%d" % (L, ovh))
 
 
+def test_arrays_that_start_on_odd_8_byte_boundaries():
+    """Input arrays that are views starting 8 bytes into an allocation (so 16-byte loads cannot
+    start at their first element), for batches whose slices touch both ends of the arrays."""
+    for name, count in (("large", 40), ("sweep", 70), ("divergence", 300), ("pr1", 1)):
+        w = taskgen.WORKLOADS[name]
+        b = w.generate(11, count)
+        tens = {}
+        for f, arr in b.arrays().items():
+            for shift in (1,):
+                pad = torch.full((arr.shape[0] + 3,), (1 << 62) + 12345, dtype=torch.int64, device="cuda")
+                pad[shift:shift + arr.shape[0]] = torch.from_numpy(arr).cuda()
+                tens[f] = pad[shift:shift + arr.shape[0]]
+        ts = binding.DeviceTasksets(tens)
+        for policy in MODES4:
+            w_ref, s_ref, _ = rta.analyse(b, policy, w.timeslice_us, w.overhead_us)
+            wc, sc = binding.rta_batch(ts, policy, w.timeslice_us, w.overhead_us)
+            torch.cuda.synchronize()
+            assert (sc.cpu().numpy() == s_ref).all() and (wc.cpu().numpy() == w_ref).all(), (name, policy)
+
+
 def test_determinism_and_output_reuse():
     b = taskgen.WORKLOADS["divergence"].generate(1000, 4000)
     ts = binding.DeviceTasksets.from_host(b)
