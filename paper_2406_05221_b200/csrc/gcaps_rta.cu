@@ -399,10 +399,16 @@ __host__ __device__ __forceinline__ void make_reciprocal(u32 d, u32 &magic, u32 
   const int k = (28 + s) > 32 ? (28 + s) : 32;
   shift = (u32)(k - 32);
 #ifdef __CUDA_ARCH__
-  // estimate 2^k / d in double precision (error far below 1), then make it exact with integers
-  const double two_k = __hiloint2double((1023 + k) << 20, 0);
-  u32 q = __double2uint_rd(two_k * __drcp_rn((double)d));
-  i64 rem = (i64)(1ull << k) - (i64)((u64)q * d);
+  // estimate 2^k / d in single precision (off by less than 2^10), correct the estimate once with
+  // the same approximate reciprocal (off by at most 1 then), and finish with integers.  Checked
+  // against the exact quotient for every d in [2, 2^26), also with the reciprocal off by 8 ulp.
+  float inv;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(__uint2float_rn(d)));
+  const u32 q0 = __float2uint_rd(inv * __int_as_float((127 + k) << 23));
+  const i64 rem0 = (i64)(1ull << k) - (i64)((u64)q0 * d);
+  const int c = __float2int_rd(__ll2float_rn(rem0) * inv);
+  u32 q = q0 + (u32)c;
+  i64 rem = rem0 - (i64)c * (i64)d;
   if (rem < 0) {
     q -= 1;
     rem += d;
@@ -479,7 +485,7 @@ struct FastLayout {
   static constexpr int MAXN = 32 * SLOTS;
   // a prefix array takes slices of up to CAP-1 elements and is written 128 words at a time
   static constexpr int CAP = (6 * MAXN + 127) / 128 * 128;
-  static constexpr int kInfo = 0;  // uint4 per rank: deadline, base, core, position | GPU flag
+  static constexpr int kInfo = 0;  // uint4 per rank: deadline, core, base, position | GPU flag
   static constexpr int kQ0 = 4 * MAXN + 4;
   static constexpr int kQ1 = kQ0 + CAP + 4;
   static constexpr int kFastWords = kQ1 + CAP;
@@ -560,15 +566,15 @@ template <int SLOTS, int MODE>
 __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane) {
   typedef FastLayout<SLOTS> Lay;
   constexpr int MAXN = Lay::MAXN, CAP = Lay::CAP;
-  constexpr int BC = SLOTS <= 4 ? SLOTS : 4;  // 128-element steps whose loads are issued together
-  constexpr int BG = SLOTS <= 2 ? SLOTS : 2;
+  constexpr int BC = SLOTS <= 2 ? SLOTS : 2;  // 128-element steps whose loads are issued together
+  constexpr int BG = 1;
   constexpr bool kGcaps = MODE < 2;
   const bool literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
   uint4 *info = reinterpret_cast<uint4 *>(buf + Lay::kInfo);
   u32 *Q0 = buf + Lay::kQ0, *Q1 = buf + Lay::kQ1;
 
   // ---- stage: per-task scalars, lane = position; rank ----------------------------------------
-  u32 T[SLOTS], D[SLOTS], core[SLOTS];
+  u32 T[SLOTS];
   int rank[SLOTS], c0[SLOTS], g0[SLOTS];
   bool ok = true;
   int Nc, Ng;
@@ -590,6 +596,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       return false;
     Nc = (int)Nc64, Ng = (int)Ng64;
     u32 high = 0;  // any set bit: some value does not fit the 32-bit path
+    u32 D[SLOTS], core[SLOTS];
     int prio[SLOTS];
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
@@ -648,6 +655,11 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
         rank[s] = i < n ? r : MAXN;
       }
     }
+    // what every lane must know about the task of a given rank (base and GPU flag follow)
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s)
+      if (lane + 32 * s < n)
+        *reinterpret_cast<uint2 *>(&info[rank[s]]) = make_uint2(D[s], core[s]);
   }
   // end offsets: the next task's start (positions beyond n hold the total)
   int c1[SLOTS], g1[SLOTS];
@@ -776,20 +788,21 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     if (lane + 32 * s < n) {
-      info[rank[s]] = make_uint4(D[s], base[s], core[s], (u32)(lane + 32 * s) | (eta[s] > 0 ? 0x10000u : 0u));
+      *(reinterpret_cast<uint2 *>(&info[rank[s]]) + 1) =
+          make_uint2(base[s], (u32)(lane + 32 * s) | (eta[s] > 0 ? 0x10000u : 0u));
       xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], S[s]);
     }
   }
   __syncwarp();
-  u32 Tm1[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS];
+  u32 Tm1[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS], core[SLOTS];
   bool gpu[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + 32 * s;
     const uint4 x = r < n ? xch[r] : make_uint4(2u, 0u, 0u, 0u);
-    const uint4 f = r < n ? info[r] : make_uint4(0u, 0u, 0xffffffffu, 0u);
+    const uint4 f = r < n ? info[r] : make_uint4(0u, 0xffffffffu, 0u, 0u);
     Tm1[s] = x.x - 1, A[s] = x.y, Ge[s] = x.z, S[s] = x.w;
-    core[s] = f.z, pos_of[s] = f.w & 0xffffu, gpu[s] = (f.w & 0x10000u) != 0;
+    core[s] = f.y, pos_of[s] = f.w & 0xffffu, gpu[s] = (f.w & 0x10000u) != 0;
     if (MODE == 0) {
       Wa[s] = A[s] + (gpu[s] ? S[s] : 0u);  // Lemma 15: C_h, or C_h + G^{m*}_h
       Wb[s] = gpu[s] ? Ge[s] + S[s] : 0u;   // Lemma 13, other cores: G^{e*}_h
@@ -804,14 +817,14 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
 
   // ---- iterate in rank order ------------------------------------------------------------------
   u32 magic[SLOTS], shift[SLOTS];         // reciprocal of T_h, made when the slot is first needed
-  u32 Jc[SLOTS], Jg[SLOTS], Rown[SLOTS];  // jitters with T_h - 1 folded in (ceiling), own result
+  u32 Jc[SLOTS], Jg[SLOTS];               // jitters with T_h - 1 folded in (ceiling)
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Tm1[s], Rown[s] = 0, magic[s] = 0, shift[s] = 0;
+  for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Tm1[s], magic[s] = 0, shift[s] = 0;
   int n_done = n;
   int verdict = 0;
   for (int pos = 0; pos < n; ++pos) {
     const uint4 f = info[pos];
-    const u32 Di = f.x, base_i = f.y, core_i = f.z;
+    const u32 Di = f.x, core_i = f.y, base_i = f.z;
     const bool gi = (f.w & 0x10000u) != 0;
     const int smax = (pos - 1) >> 5;  // -1 for the first task: nothing interferes
     if ((pos & 31) == 1) {            // the first task that looks at slot smax
@@ -888,24 +901,23 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       verdict = v;
       break;
     }
-    // publish: the owner keeps R_i and its jitters J^c = R - (C+G^m), J^g = R - G^e (a CPU-only
-    // task has no J^c unless the printed form of Lemma 7 is asked for)
+    // publish: the owner writes R_i and forms its jitters J^c = R - (C+G^m), J^g = R - G^e (a
+    // CPU-only task has no J^c unless the printed form of Lemma 7 is asked for)
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
       if (lane + 32 * s == pos) {
-        Rown[s] = R;
+        p.out_wcrt[a + pos_of[s]] = (i64)R;
         if (MODE == 0 ? gpu[s] : (MODE == 2 ? (gpu[s] || literal) : false)) Jc[s] = R - A[s] + Tm1[s];
         Jg[s] = R - Ge[s] + Tm1[s];
       }
     }
   }
-  // ---- write ----------------------------------------------------------------------------------
+  // ---- write the sentinels of the tasks that did not converge ---------------------------------
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + 32 * s;
-    if (r < n)
-      p.out_wcrt[a + pos_of[s]] =
-          r < n_done ? (i64)Rown[s] : (r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED);
+    if (r < n && r >= n_done)
+      p.out_wcrt[a + pos_of[s]] = r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED;
   }
   if (lane == 0) p.out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
   __syncwarp();
@@ -916,55 +928,71 @@ __device__ __forceinline__ void prefetch_l2(const void *ptr) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
 }
 
-// What a warp knows in advance about one taskset of its chunk.
+// What a warp knows in advance about one taskset of a chunk (kept in shared memory).
 struct Ahead {
   i64 t, a;        // taskset index, first task
   i64 c_lo, g_lo;  // first CPU segment, first GPU segment
   int n, nc, ng;   // tasks, CPU segments, GPU segments; nc = ng = 0 unless safe to prefetch
   int pf;          // 1 if the task range is one the fast path could take
 };
+constexpr int kMaxChunk = 8;
+constexpr int kAheadWords = 2 * kMaxChunk * (int)(sizeof(Ahead) / sizeof(u32));  // two chunks
 
 // Persistent launch over one size bin: warps pull chunks of tasksets from the bin's counter.
 // While one taskset is analysed the input of the next one is already on its way into L2.
+// blocks per SM the register allocation aims at: more warps in flight matter more here than a
+// few spilled values, because every phase is a chain of dependent instructions
+__host__ __device__ constexpr int min_blocks(int slots) {
+  return slots <= 3 ? 6 : slots == 4 ? 4 : slots == 6 ? 3 : 2;
+}
+
 template <int SLOTS, int MODE>
-__global__ void __launch_bounds__(kBlockThreads) rta_kernel(KParams p, int bin) {
+__global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(KParams p, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   typedef FastLayout<SLOTS> Lay;
   constexpr int MAXN = 32 * SLOTS;
-  constexpr int kChunk = 4;  // tasksets per pull
+  constexpr int kWarpWords = Lay::kWords + kAheadWords;
   static_assert(sizeof(GroupSmem<MAXN>) <= sizeof(u32) * Lay::kWords, "exact path fits");
   static_assert(6 * MAXN <= Lay::CAP, "prefetched ranges are ranges the fast path accepts");
+  static_assert(kWarpWords % 4 == 0 && sizeof(Ahead) % 16 == 0, "alignment");
   const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * Lay::kWords;
+  u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * kWarpWords;
+  Ahead *ahead = reinterpret_cast<Ahead *>(buf + Lay::kWords);  // [2][kMaxChunk]
   const unsigned int start = p.hdr->bin_start[bin], count = p.hdr->bin_count[bin];
   const bool fast_call = p.ovh < (1 << 20);  // keeps 2*eps*eta and (eta+1)*eps in 32 bits
+  // tasksets per pull: 8 when the bin is large, fewer when it would leave warps without work
+  const unsigned int n_warps = gridDim.x * (kBlockThreads / 32);
+  const int kChunk = count >= 32 * n_warps ? kMaxChunk : (count >= 8 * n_warps ? 4 : 1);
 
-  // lanes 0..kChunk-1 each look up one taskset of a chunk
-  auto look_up = [&](unsigned int first, Ahead &me) {
-    me.t = 0, me.a = 0, me.c_lo = me.g_lo = 0, me.n = me.nc = me.ng = 0, me.pf = 0;
-    if (lane < kChunk && first < count && first + lane < count) {
-      me.t = (i64)p.perm[start + first + lane];
-      me.a = p.task_off[me.t] - p.task_base;
-      const i64 b = p.task_off[me.t + 1] - p.task_base;
-      if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN) {
-        me.pf = 1, me.n = (int)(b - me.a);
-        me.c_lo = p.cseg_off[me.a] - p.cseg_base, me.g_lo = p.gseg_off[me.a] - p.gseg_base;
-        const i64 c_hi = p.cseg_off[b] - p.cseg_base, g_hi = p.gseg_off[b] - p.gseg_base;
-        if (me.c_lo >= 0 && c_hi <= p.n_csegs && c_hi - me.c_lo <= 6 * MAXN && c_hi > me.c_lo)
-          me.nc = (int)(c_hi - me.c_lo);
-        if (me.g_lo >= 0 && g_hi <= p.n_gsegs && g_hi - me.g_lo <= 6 * MAXN && g_hi > me.g_lo)
-          me.ng = (int)(g_hi - me.g_lo);
+  // lanes 0..kChunk-1 each look up one taskset of a chunk and leave what they found in `slot`
+  auto look_up = [&](unsigned int first, Ahead *slot) {
+    if (lane < kChunk) {
+      Ahead me;
+      me.t = 0, me.a = 0, me.c_lo = me.g_lo = 0, me.n = me.nc = me.ng = 0, me.pf = 0;
+      if (first < count && first + lane < count) {
+        me.t = (i64)p.perm[start + first + lane];
+        me.a = p.task_off[me.t] - p.task_base;
+        const i64 b = p.task_off[me.t + 1] - p.task_base;
+        if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN) {
+          me.pf = 1, me.n = (int)(b - me.a);
+          me.c_lo = p.cseg_off[me.a] - p.cseg_base, me.g_lo = p.gseg_off[me.a] - p.gseg_base;
+          const i64 c_hi = p.cseg_off[b] - p.cseg_base, g_hi = p.gseg_off[b] - p.gseg_base;
+          if (me.c_lo >= 0 && c_hi <= p.n_csegs && c_hi - me.c_lo <= 6 * MAXN && c_hi > me.c_lo)
+            me.nc = (int)(c_hi - me.c_lo);
+          if (me.g_lo >= 0 && g_hi <= p.n_gsegs && g_hi - me.g_lo <= 6 * MAXN && g_hi > me.g_lo)
+            me.ng = (int)(g_hi - me.g_lo);
+        }
       }
+      slot[lane] = me;
     }
+    __syncwarp();
   };
-  // all lanes: pull the lines of taskset c of the chunk towards L2 (16 elements per line; only
-  // addresses inside the arrays are named)
-  auto prefetch = [&](const Ahead &me, int c) {
-    if (__shfl_sync(kFull, me.pf, c) == 0) return;
-    const i64 a = __shfl_sync(kFull, me.a, c);
-    const i64 c_lo = __shfl_sync(kFull, me.c_lo, c), g_lo = __shfl_sync(kFull, me.g_lo, c);
-    const int n = __shfl_sync(kFull, me.n, c), nc = __shfl_sync(kFull, me.nc, c);
-    const int ng = __shfl_sync(kFull, me.ng, c);
+  // all lanes: pull the lines of a taskset towards L2 (16 elements per line; only addresses
+  // inside the arrays are named)
+  auto prefetch = [&](const Ahead &me) {
+    if (me.pf == 0) return;
+    const i64 a = me.a, c_lo = me.c_lo, g_lo = me.g_lo;
+    const int n = me.n, nc = me.nc, ng = me.ng;
     for (int e = 16 * lane; e < n; e += 16 * 32) {
       prefetch_l2(p.period + a + e), prefetch_l2(p.deadline + a + e), prefetch_l2(p.priority + a + e);
       prefetch_l2(p.core + a + e), prefetch_l2(p.cseg_off + a + e), prefetch_l2(p.gseg_off + a + e);
@@ -977,27 +1005,26 @@ __global__ void __launch_bounds__(kBlockThreads) rta_kernel(KParams p, int bin) 
   unsigned int first = 0;
   if (lane == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
   first = __shfl_sync(kFull, first, 0);
-  Ahead cur;
-  look_up(first, cur);
-  if (first < count) prefetch(cur, 0);
+  int which = 0;
+  look_up(first, ahead);
+  if (first < count) prefetch(ahead[0]);
   while (first < count) {
     unsigned int nfirst = 0;
     if (lane == 0) nfirst = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
-    Ahead nxt;
-    nxt.t = 0, nxt.a = 0, nxt.c_lo = nxt.g_lo = 0, nxt.n = nxt.nc = nxt.ng = 0, nxt.pf = 0;
+    const Ahead *cur = ahead + which * kMaxChunk;
+    Ahead *nxt = ahead + (which ^ 1) * kMaxChunk;
     const int in_chunk = count - first < (unsigned int)kChunk ? (int)(count - first) : kChunk;
     for (int c = 0; c < in_chunk; ++c) {
-      if (c + 1 < in_chunk) prefetch(cur, c + 1);
+      if (c + 1 < in_chunk) prefetch(cur[c + 1]);
       if (c == 1 || in_chunk == 1) {  // the next chunk's index has arrived by now
         nfirst = __shfl_sync(kFull, nfirst, 0);
         look_up(nfirst, nxt);
       }
-      if (c == in_chunk - 1 && nfirst < count) prefetch(nxt, 0);
-      const i64 t = __shfl_sync(kFull, cur.t, c), a = __shfl_sync(kFull, cur.a, c);
-      const int n = __shfl_sync(kFull, cur.n, c);
+      if (c == in_chunk - 1 && nfirst < count) prefetch(nxt[0]);
+      const i64 t = cur[c].t, a = cur[c].a;
+      const int n = cur[c].n;
       bool done = false;
-      if (fast_call && __shfl_sync(kFull, cur.pf, c) != 0)
-        done = analyse_fast<SLOTS, MODE>(p, t, a, n, buf, lane);
+      if (fast_call && cur[c].pf != 0) done = analyse_fast<SLOTS, MODE>(p, t, a, n, buf, lane);
       __syncwarp();
       if (!done) {
         // the exact path reads task_off again and validates everything itself
@@ -1006,7 +1033,7 @@ __global__ void __launch_bounds__(kBlockThreads) rta_kernel(KParams p, int bin) 
       __syncwarp();
     }
     first = nfirst;
-    cur = nxt;
+    which ^= 1;
   }
 }
 
@@ -1136,7 +1163,7 @@ void fill_params(KParams *p, const gcaps_tasksets_t *ts, int64_t n_tasksets, int
 template <int SLOTS, int MODE>
 cudaError_t launch_bin(const KParams &p, int bin, int sm_count, cudaStream_t st) {
   constexpr int kWarps = kBlockThreads / 32;
-  const size_t smem = sizeof(u32) * FastLayout<SLOTS>::kWords * kWarps;
+  const size_t smem = sizeof(u32) * (FastLayout<SLOTS>::kWords + kAheadWords) * kWarps;
   static int blocks_per_sm[64] = {0};  // per device; 0 = not set up yet
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);

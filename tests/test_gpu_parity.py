@@ -212,6 +212,30 @@ def test_values_around_the_32_bit_path_limit():
             assert_parity(b, policy, L, ovh, "limit L=%d ovh=%d" % (L, ovh))
 
 
+def test_every_class_of_period_as_a_divisor():
+    """The kernels divide by each interferer's period with a precomputed reciprocal.  Periods of
+    every magnitude (powers of two and their neighbours, small values, random ones up to the
+    32-bit path's limit) against dividends from a few thousand up to 2^26."""
+    rng = np.random.default_rng(33)
+    lim = 1 << 26
+    periods = [2, 3, 4, 5, 6, 7, 8, 9, 15, 16, 17, 31, 33, 1000, 1023, 1024, 1025]
+    periods += [(1 << k) + d for k in range(5, 26) for d in (-1, 0, 1)]
+    periods += [lim - 1, lim - 2, lim - 3] + [int(x) for x in rng.integers(2, lim, 3000)]
+    periods += [int(x) for x in np.exp(rng.uniform(np.log(2), np.log(lim), 3000))]
+    sets = []
+    for T in periods:
+        T = max(2, min(lim - 1, T))
+        own = int(rng.choice([5000, 1 << 20, 1 << 25]))
+        ch = max(1, T // int(rng.integers(3, 9)))
+        sets.append([dict(T=T, prio=3, core=0, cseg=[ch]),
+                     dict(T=max(2, T // 2 + 1), prio=2, core=1, cseg=[1], gseg=[(0, max(1, T // 7))]),
+                     dict(T=lim - 1, prio=1, core=0, cseg=[own], gseg=[(1, 1)])])
+    b = batch_of(sets)
+    for policy in MODES4:
+        w, s = assert_parity(b, policy, 1024, 0, "divisors")
+    assert (w[2::3] > 0).mean() > 0.5   # most of the low-priority tasks converge (many sweeps)
+
+
 def test_arrays_that_start_on_odd_8_byte_boundaries():
     """Input arrays that are views starting 8 bytes into an allocation (so 16-byte loads cannot
     start at their first element), for batches whose slices touch both ends of the arrays."""
