@@ -924,28 +924,24 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   return true;
 }
 
-__device__ __forceinline__ void prefetch_l2(const void *ptr) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
-}
-
 // What a warp knows in advance about one taskset of a chunk (kept in shared memory).
 struct Ahead {
-  i64 t, a;        // taskset index, first task
-  i64 c_lo, g_lo;  // first CPU segment, first GPU segment
-  int n, nc, ng;   // tasks, CPU segments, GPU segments; nc = ng = 0 unless safe to prefetch
-  int pf;          // 1 if the task range is one the fast path could take
+  i64 t, a;  // taskset index, first task
+  int n;     // tasks
+  int fast;  // 1 if the task range is one the 32-bit path could take
 };
 constexpr int kMaxChunk = 8;
 constexpr int kAheadWords = 2 * kMaxChunk * (int)(sizeof(Ahead) / sizeof(u32));  // two chunks
 
-// Persistent launch over one size bin: warps pull chunks of tasksets from the bin's counter.
-// While one taskset is analysed the input of the next one is already on its way into L2.
 // blocks per SM the register allocation aims at: more warps in flight matter more here than a
-// few spilled values, because every phase is a chain of dependent instructions
+// few spilled values, because every phase is a chain of dependent instructions and the loads of
+// a taskset can only be hidden behind the work of other warps
 __host__ __device__ constexpr int min_blocks(int slots) {
   return slots <= 3 ? 6 : slots == 4 ? 4 : slots == 6 ? 3 : 2;
 }
 
+// Persistent launch over one size bin: warps pull chunks of tasksets from the bin's counter; the
+// index and task range of the next chunk are fetched while the current one is analysed.
 template <int SLOTS, int MODE>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(KParams p, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -953,8 +949,7 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(K
   constexpr int MAXN = 32 * SLOTS;
   constexpr int kWarpWords = Lay::kWords + kAheadWords;
   static_assert(sizeof(GroupSmem<MAXN>) <= sizeof(u32) * Lay::kWords, "exact path fits");
-  static_assert(6 * MAXN <= Lay::CAP, "prefetched ranges are ranges the fast path accepts");
-  static_assert(kWarpWords % 4 == 0 && sizeof(Ahead) % 16 == 0, "alignment");
+  static_assert(kWarpWords % 4 == 0 && sizeof(Ahead) % 8 == 0, "alignment");
   const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
   u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(buf + Lay::kWords);  // [2][kMaxChunk]
@@ -968,38 +963,17 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(K
   auto look_up = [&](unsigned int first, Ahead *slot) {
     if (lane < kChunk) {
       Ahead me;
-      me.t = 0, me.a = 0, me.c_lo = me.g_lo = 0, me.n = me.nc = me.ng = 0, me.pf = 0;
+      me.t = 0, me.a = 0, me.n = 0, me.fast = 0;
       if (first < count && first + lane < count) {
         me.t = (i64)p.perm[start + first + lane];
         me.a = p.task_off[me.t] - p.task_base;
         const i64 b = p.task_off[me.t + 1] - p.task_base;
-        if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN) {
-          me.pf = 1, me.n = (int)(b - me.a);
-          me.c_lo = p.cseg_off[me.a] - p.cseg_base, me.g_lo = p.gseg_off[me.a] - p.gseg_base;
-          const i64 c_hi = p.cseg_off[b] - p.cseg_base, g_hi = p.gseg_off[b] - p.gseg_base;
-          if (me.c_lo >= 0 && c_hi <= p.n_csegs && c_hi - me.c_lo <= 6 * MAXN && c_hi > me.c_lo)
-            me.nc = (int)(c_hi - me.c_lo);
-          if (me.g_lo >= 0 && g_hi <= p.n_gsegs && g_hi - me.g_lo <= 6 * MAXN && g_hi > me.g_lo)
-            me.ng = (int)(g_hi - me.g_lo);
-        }
+        if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN)
+          me.fast = 1, me.n = (int)(b - me.a);
       }
       slot[lane] = me;
     }
     __syncwarp();
-  };
-  // all lanes: pull the lines of a taskset towards L2 (16 elements per line; only addresses
-  // inside the arrays are named)
-  auto prefetch = [&](const Ahead &me) {
-    if (me.pf == 0) return;
-    const i64 a = me.a, c_lo = me.c_lo, g_lo = me.g_lo;
-    const int n = me.n, nc = me.nc, ng = me.ng;
-    for (int e = 16 * lane; e < n; e += 16 * 32) {
-      prefetch_l2(p.period + a + e), prefetch_l2(p.deadline + a + e), prefetch_l2(p.priority + a + e);
-      prefetch_l2(p.core + a + e), prefetch_l2(p.cseg_off + a + e), prefetch_l2(p.gseg_off + a + e);
-    }
-    for (int e = 16 * lane; e < nc; e += 16 * 32) prefetch_l2(p.cseg_wcet + c_lo + e);
-    for (int e = 16 * lane; e < ng; e += 16 * 32)
-      prefetch_l2(p.gseg_misc + g_lo + e), prefetch_l2(p.gseg_exec + g_lo + e);
   };
 
   unsigned int first = 0;
@@ -1007,7 +981,6 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(K
   first = __shfl_sync(kFull, first, 0);
   int which = 0;
   look_up(first, ahead);
-  if (first < count) prefetch(ahead[0]);
   while (first < count) {
     unsigned int nfirst = 0;
     if (lane == 0) nfirst = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
@@ -1015,16 +988,14 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(K
     Ahead *nxt = ahead + (which ^ 1) * kMaxChunk;
     const int in_chunk = count - first < (unsigned int)kChunk ? (int)(count - first) : kChunk;
     for (int c = 0; c < in_chunk; ++c) {
-      if (c + 1 < in_chunk) prefetch(cur[c + 1]);
       if (c == 1 || in_chunk == 1) {  // the next chunk's index has arrived by now
         nfirst = __shfl_sync(kFull, nfirst, 0);
         look_up(nfirst, nxt);
       }
-      if (c == in_chunk - 1 && nfirst < count) prefetch(nxt[0]);
       const i64 t = cur[c].t, a = cur[c].a;
       const int n = cur[c].n;
       bool done = false;
-      if (fast_call && cur[c].pf != 0) done = analyse_fast<SLOTS, MODE>(p, t, a, n, buf, lane);
+      if (fast_call && cur[c].fast != 0) done = analyse_fast<SLOTS, MODE>(p, t, a, n, buf, lane);
       __syncwarp();
       if (!done) {
         // the exact path reads task_off again and validates everything itself
