@@ -926,10 +926,15 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
 
 // What a warp knows in advance about one taskset of a chunk (kept in shared memory).
 struct Ahead {
-  i64 t, a;  // taskset index, first task
-  int n;     // tasks
-  int fast;  // 1 if the task range is one the 32-bit path could take
+  i64 t, a;        // taskset index, first task
+  i64 c_lo, g_lo;  // first CPU segment, first GPU segment
+  int n, nc, ng;   // tasks, CPU segments, GPU segments (nc = ng = 0 unless the ranges are sound)
+  int fast;        // 1 if the task range is one the 32-bit path could take
 };
+
+__device__ __forceinline__ void prefetch_l2(const void *ptr) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
 constexpr int kMaxChunk = 8;
 constexpr int kAheadWords = 2 * kMaxChunk * (int)(sizeof(Ahead) / sizeof(u32));  // two chunks
 
@@ -949,7 +954,7 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(K
   constexpr int MAXN = 32 * SLOTS;
   constexpr int kWarpWords = Lay::kWords + kAheadWords;
   static_assert(sizeof(GroupSmem<MAXN>) <= sizeof(u32) * Lay::kWords, "exact path fits");
-  static_assert(kWarpWords % 4 == 0 && sizeof(Ahead) % 8 == 0, "alignment");
+  static_assert(kWarpWords % 4 == 0 && sizeof(Ahead) % 16 == 0, "alignment");
   const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
   u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(buf + Lay::kWords);  // [2][kMaxChunk]
@@ -963,13 +968,20 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(K
   auto look_up = [&](unsigned int first, Ahead *slot) {
     if (lane < kChunk) {
       Ahead me;
-      me.t = 0, me.a = 0, me.n = 0, me.fast = 0;
+      me.t = 0, me.a = 0, me.c_lo = me.g_lo = 0, me.n = me.nc = me.ng = 0, me.fast = 0;
       if (first < count && first + lane < count) {
         me.t = (i64)p.perm[start + first + lane];
         me.a = p.task_off[me.t] - p.task_base;
         const i64 b = p.task_off[me.t + 1] - p.task_base;
-        if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN)
+        if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN) {
           me.fast = 1, me.n = (int)(b - me.a);
+          me.c_lo = p.cseg_off[me.a] - p.cseg_base, me.g_lo = p.gseg_off[me.a] - p.gseg_base;
+          const i64 c_hi = p.cseg_off[b] - p.cseg_base, g_hi = p.gseg_off[b] - p.gseg_base;
+          if (me.c_lo >= 0 && c_hi <= p.n_csegs && c_hi - me.c_lo < Lay::CAP && c_hi > me.c_lo)
+            me.nc = (int)(c_hi - me.c_lo);
+          if (me.g_lo >= 0 && g_hi <= p.n_gsegs && g_hi - me.g_lo < Lay::CAP && g_hi > me.g_lo)
+            me.ng = (int)(g_hi - me.g_lo);
+        }
       }
       slot[lane] = me;
     }
@@ -994,6 +1006,15 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(K
       }
       const i64 t = cur[c].t, a = cur[c].a;
       const int n = cur[c].n;
+      {  // the segment slices start their way into L2 now; the per-task loads follow at once, so
+         // that the running sums later wait for L2 rather than for DRAM (16 elements per line,
+         // only addresses inside the arrays)
+        const i64 c_lo = cur[c].c_lo, g_lo = cur[c].g_lo;
+        const int nc = cur[c].nc, ng = cur[c].ng;
+        for (int e = 16 * lane; e < nc; e += 16 * 32) prefetch_l2(p.cseg_wcet + c_lo + e);
+        for (int e = 16 * lane; e < ng; e += 16 * 32)
+          prefetch_l2(p.gseg_misc + g_lo + e), prefetch_l2(p.gseg_exec + g_lo + e);
+      }
       bool done = false;
       if (fast_call && cur[c].fast != 0) done = analyse_fast<SLOTS, MODE>(p, t, a, n, buf, lane);
       __syncwarp();
