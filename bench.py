@@ -33,6 +33,30 @@ ALU_PEAK_LANEOPS = 148 * 128 * 1.965e9
 K_TERM, K_SETUP = 6, 16   # algorithmic integer lane-operations per interference term / per task
 # kernels launched by one gcaps_rta_batch call: 3 plan kernels + one analysis kernel per size bin
 LAUNCHES_PER_CALL = 9
+# DRAM bytes (read + write) per taskset of the analysis kernel on the 'large' workload, from the
+# ncu capture summarised in profiles/rta_kernel_large_131072_full.md (131,072 tasksets; traffic
+# grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
+# the one the counters were taken from.
+CAPTURED_TRAFFIC = {
+    "source_sha256": "67e44d64fddf7bb10de66faf9b1edb1ec1bec845cf8031533a748abc9cd61e33",
+    "workload": "large",
+    "bytes_per_taskset": {"gcaps": (1247331000 + 82918656) / 131072.0,
+                          "rr": (1245120000 + 81220608) / 131072.0},
+}
+
+
+def captured_traffic(workload_name, policy_name, tasksets):
+    """DRAM traffic of one analysis launch, or None if the capture does not apply any more."""
+    import hashlib
+    src = os.path.join(ROOT, "paper_2406_05221_b200", "csrc", "gcaps_rta.cu")
+    try:
+        with open(src, "rb") as fh:
+            digest = hashlib.sha256(fh.read()).hexdigest()
+    except OSError:
+        return None
+    if digest != CAPTURED_TRAFFIC["source_sha256"] or workload_name != CAPTURED_TRAFFIC["workload"]:
+        return None
+    return CAPTURED_TRAFFIC["bytes_per_taskset"][policy_name] * tasksets
 
 
 def measured_peaks():
@@ -271,7 +295,9 @@ def main():
         dom = int(np.argmax(per_policy_ms))
         achieved = bytes_per_call / (per_policy_ms[dom] * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
+                "frac": achieved / peak,
+                "traffic": captured_traffic(workload.name, names[dom], count),
+                "peak_kind": peak_kind,
                 "kernel": "analysis kernel of the %s call (the call's plan kernels are inside the timing)"
                           % names[dom].upper(),
                 "algorithmic_bytes_per_launch": bytes_per_call,
