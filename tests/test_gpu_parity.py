@@ -331,3 +331,70 @@ def test_full_size_large_workload_sampled():
         D = b.deadline.reshape(-1, 80)
         ok = wc >= 0
         assert (wc[ok] <= D[ok]).all()
+
+
+def _sampled_parity(batch, ts, policy, L, ovh, rng, n_sample, what):
+    """Runs the library on the whole device batch and the oracle on a random sample of tasksets."""
+    wc, sc = binding.rta_batch(ts, policy, L, ovh)
+    torch.cuda.synchronize()
+    wc, sc = wc.cpu().numpy(), sc.cpu().numpy()
+    sample = np.sort(rng.choice(batch.n_tasksets, min(n_sample, batch.n_tasksets), replace=False))
+    sub = batch.select(sample)
+    w_ref, s_ref, _ = rta.analyse(sub, policy, L, ovh)
+    assert (sc[sample] == s_ref).all(), what
+    pos = np.concatenate([np.arange(batch.task_off[t], batch.task_off[t + 1]) for t in sample])
+    assert (wc[pos] == w_ref).all(), what
+    # properties that hold at any size
+    assert sc.max() <= 1, what
+    first = batch.task_off[:-1]
+    nonempty = np.diff(batch.task_off) > 0
+    has_neg = np.zeros(batch.n_tasksets, bool)
+    has_neg[nonempty] = np.minimum.reduceat(wc, first[nonempty]) < 0
+    assert ((sc == 1) == ~has_neg).all(), what
+    ok = wc >= 0
+    assert (wc[ok] <= batch.deadline[ok]).all(), what
+    return sc
+
+
+def test_full_size_schedulability_sweep_sampled():
+    """All nine points of the utilisation sweep at 100,000 tasksets each, both policies."""
+    w = taskgen.WORKLOADS["sweep"]
+    rng = np.random.default_rng(17)
+    ratio = {0: [], 1: []}
+    for stream in range(len(w.streams)):
+        b = w.generate(0, w.n_tasksets, stream=stream)
+        ts = binding.DeviceTasksets.from_host(b)
+        for policy in (0, 1):
+            sc = _sampled_parity(b, ts, policy, w.timeslice_us, w.overhead_us, rng, 700,
+                                 "sweep point %d policy %d" % (stream, policy))
+            ratio[policy].append(float((sc == 1).mean()))
+    # schedulability falls as the utilisation per core rises, and GCAPS stays above round robin
+    for policy in (0, 1):
+        assert ratio[policy][0] >= ratio[policy][-1]
+    assert ratio[0][0] > 0.9 and ratio[0][0] > ratio[1][0]
+
+
+def test_full_size_rr_driver_model_sweep_sampled():
+    """200,000 tasksets under round robin for all 25 (time slice, context switch) pairs."""
+    w = taskgen.WORKLOADS["rr_model"]
+    rng = np.random.default_rng(18)
+    b = w.generate(0, w.n_tasksets)
+    ts = binding.DeviceTasksets.from_host(b)
+    for L in w.timeslices:
+        for theta in w.overheads:
+            _sampled_parity(b, ts, 1, L, theta, rng, 300, "rr model L=%d theta=%d" % (L, theta))
+
+
+def test_full_size_divergence_stress_sampled():
+    """The 10,000,000-taskset divergence workload in chunks of 1,000,000, both policies."""
+    w = taskgen.WORKLOADS["divergence"]
+    rng = np.random.default_rng(19)
+    chunk = 1_000_000
+    for first in range(0, w.n_tasksets, chunk):
+        b = w.generate(first, chunk)
+        ts = binding.DeviceTasksets.from_host(b)
+        for policy in (0, 1):
+            _sampled_parity(b, ts, policy, w.timeslice_us, w.overhead_us, rng, 400,
+                            "divergence chunk %d policy %d" % (first // chunk, policy))
+        del ts
+        torch.cuda.empty_cache()
