@@ -157,6 +157,20 @@ int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int pol
                          uint8_t *out_sched);
 
 /*
+ * gcaps_rta_batch_host_multi -- gcaps_rta_batch_host for several analyses of the same batch (the
+ * paper's experiments run every taskset through GCAPS and through round robin, Sec. 7.1): the
+ * inputs cross the host-device link once per chunk and are analysed n_policies times on the
+ * device.  policies[q] is a GCAPS_POLICY_* | flags word, 1 <= n_policies <=
+ * GCAPS_RTA_MAX_HOST_POLICIES; out_wcrt[q] / out_sched[q] are the host arrays of analysis q
+ * ([ts->n_tasks] and [n_tasksets]).  timeslice_us and ctx_switch_overhead_us apply to all of
+ * them.  Same return codes and synchronous behaviour as gcaps_rta_batch_host.
+ */
+#define GCAPS_RTA_MAX_HOST_POLICIES 8
+int gcaps_rta_batch_host_multi(const gcaps_tasksets_t *ts, int64_t n_tasksets, const int *policies,
+                               int n_policies, int64_t timeslice_us, int64_t ctx_switch_overhead_us,
+                               int64_t *const *out_wcrt, uint8_t *const *out_sched);
+
+/*
  * gcaps_rta_batch_static -- gcaps_rta_batch for callers that are not able to allocate device
  * memory.  (The paper has no counterpart: this is a convenience of this library, not a step of
  * the analysis.)

@@ -30,7 +30,8 @@ STATIC_MAX_TASKSETS = 65536
 
 EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host",
            "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
-           "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static")
+           "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static",
+           "gcaps_rta_batch_host_multi")
 
 _p64 = ctypes.POINTER(ctypes.c_int64)
 
@@ -74,6 +75,11 @@ def load_library(path: Optional[str] = None):
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
             ctypes.c_void_p, ctypes.c_void_p]
         lib.gcaps_rta_batch_host.restype = ctypes.c_int
+        lib.gcaps_rta_batch_host_multi.argtypes = [
+            ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.POINTER(ctypes.c_int), ctypes.c_int,
+            ctypes.c_int64, ctypes.c_int64, ctypes.POINTER(ctypes.c_void_p),
+            ctypes.POINTER(ctypes.c_void_p)]
+        lib.gcaps_rta_batch_host_multi.restype = ctypes.c_int
         lib.gcaps_rta_release_host.argtypes = []
         lib.gcaps_rta_release_host.restype = None
         lib.gcaps_rta_validate.argtypes = [ctypes.POINTER(CTasksets), ctypes.c_int64,
@@ -206,6 +212,26 @@ def rta_batch_host(arrays: Dict[str, np.ndarray], policy: int, timeslice_us: int
         out_sched = np.full(max(n_tasksets, 0), SCHED_INVALID, np.uint8)
     rc = lib.gcaps_rta_batch_host(ctypes.byref(c), n_tasksets, policy, timeslice_us, overhead_us,
                                   out_wcrt.ctypes.data, out_sched.ctypes.data)
+    _check(rc)
+    return out_wcrt, out_sched
+
+
+def rta_batch_host_multi(arrays: Dict[str, np.ndarray], policies, timeslice_us: int = 1024,
+                         overhead_us: int = 0, out_wcrt=None, out_sched=None):
+    """gcaps_rta_batch_host_multi: one copy of the host arrays to the device, one analysis per
+    entry of ``policies``.  Returns ``(list of out_wcrt, list of out_sched)`` numpy arrays."""
+    lib = load_library()
+    c, n_tasksets = host_struct(arrays)
+    k = len(policies)
+    if out_wcrt is None:
+        out_wcrt = [np.full(c.n_tasks, WCRT_INVALID, np.int64) for _ in range(k)]
+    if out_sched is None:
+        out_sched = [np.full(max(n_tasksets, 0), SCHED_INVALID, np.uint8) for _ in range(k)]
+    pol = (ctypes.c_int * k)(*policies)
+    pw = (ctypes.c_void_p * k)(*[a.ctypes.data for a in out_wcrt])
+    ps = (ctypes.c_void_p * k)(*[a.ctypes.data for a in out_sched])
+    rc = lib.gcaps_rta_batch_host_multi(ctypes.byref(c), n_tasksets, pol, k, timeslice_us,
+                                        overhead_us, pw, ps)
     _check(rc)
     return out_wcrt, out_sched
 

@@ -1340,10 +1340,13 @@ void gcaps_rta_release_host(void) {
   g_stage.device = -1;
 }
 
-// Copies tasksets [t, t1) (tasks [k0, k1)) to the staging slot, enqueues their analysis and the
-// copies of the results back.  The offsets of the range are known to be monotone and in range.
-static int host_chunk(const gcaps_tasksets_t *ts, int64_t t, int64_t t1, int policy, int64_t L,
-                      int64_t ovh, int64_t *out_wcrt, uint8_t *out_sched, int slot, int sm_count) {
+constexpr int kMaxHostPolicies = GCAPS_RTA_MAX_HOST_POLICIES;
+
+// Copies tasksets [t, t1) (tasks [k0, k1)) to the staging slot, enqueues their analysis under
+// every requested policy and the copies of the results back.  The offsets of the range are known to be monotone and in range.
+static int host_chunk(const gcaps_tasksets_t *ts, int64_t t, int64_t t1, const int *policies,
+                      int n_pol, int64_t L, int64_t ovh, int64_t *const *out_wcrt,
+                      uint8_t *const *out_sched, int slot, int sm_count) {
   const int64_t k0 = ts->task_off[t], k1 = ts->task_off[t1];
   const int64_t nt = t1 - t, nk = k1 - k0;
   const int64_t c0 = ts->cseg_off[k0], nc = ts->cseg_off[k1] - c0;
@@ -1357,7 +1360,9 @@ static int host_chunk(const gcaps_tasksets_t *ts, int64_t t, int64_t t1, int pol
   const size_t o_task_off = take((nt + 1) * 8), o_period = take(nk * 8), o_deadline = take(nk * 8);
   const size_t o_priority = take(nk * 8), o_core = take(nk * 8), o_cseg_off = take((nk + 1) * 8);
   const size_t o_cseg = take(nc * 8), o_gseg_off = take((nk + 1) * 8), o_gm = take(ng * 8);
-  const size_t o_ge = take(ng * 8), o_wcrt = take(nk * 8), o_sched = take(nt);
+  const size_t o_ge = take(ng * 8);
+  size_t o_wcrt[kMaxHostPolicies], o_sched[kMaxHostPolicies];
+  for (int q = 0; q < n_pol; ++q) o_wcrt[q] = take(nk * 8), o_sched[q] = take(nt);
   const size_t ws_bytes = gcaps_rta_workspace_bytes(nt);
   const size_t o_ws = take(ws_bytes);
   cudaStream_t st = g_stage.stream[slot];
@@ -1400,14 +1405,17 @@ static int host_chunk(const gcaps_tasksets_t *ts, int64_t t, int64_t t1, int pol
   dts.gseg_off = (const int64_t *)(d + o_gseg_off);
   dts.gseg_misc = (const int64_t *)(d + o_gm);
   dts.gseg_exec = (const int64_t *)(d + o_ge);
-  KParams p;
-  fill_params(&p, &dts, nt, policy, L, ovh, (int64_t *)(d + o_wcrt), d + o_sched);
-  p.task_base = k0, p.cseg_base = c0, p.gseg_base = g0;
-  int rc = enqueue_batch(p, d + o_ws, ws_bytes, sm_count, st);
-  if (rc != GCAPS_OK) return rc;
-  if (nk > 0)
-    HOST_TRY(cudaMemcpyAsync(out_wcrt + k0, d + o_wcrt, (size_t)nk * 8, cudaMemcpyDeviceToHost, st));
-  HOST_TRY(cudaMemcpyAsync(out_sched + t, d + o_sched, (size_t)nt, cudaMemcpyDeviceToHost, st));
+  for (int q = 0; q < n_pol; ++q) {  // one copy of the inputs, one analysis per policy
+    KParams p;
+    fill_params(&p, &dts, nt, policies[q], L, ovh, (int64_t *)(d + o_wcrt[q]), d + o_sched[q]);
+    p.task_base = k0, p.cseg_base = c0, p.gseg_base = g0;
+    int rc = enqueue_batch(p, d + o_ws, ws_bytes, sm_count, st);
+    if (rc != GCAPS_OK) return rc;
+    if (nk > 0)
+      HOST_TRY(cudaMemcpyAsync(out_wcrt[q] + k0, d + o_wcrt[q], (size_t)nk * 8,
+                               cudaMemcpyDeviceToHost, st));
+    HOST_TRY(cudaMemcpyAsync(out_sched[q] + t, d + o_sched[q], (size_t)nt, cudaMemcpyDeviceToHost, st));
+  }
   return GCAPS_OK;
 }
 
@@ -1426,10 +1434,23 @@ static bool host_range_is_canonical(const gcaps_tasksets_t *ts, int64_t k0, int6
 int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
                          int64_t timeslice_us, int64_t ctx_switch_overhead_us, int64_t *out_wcrt,
                          uint8_t *out_sched) {
-  int rc = check_args(ts, n_tasksets, policy, timeslice_us, ctx_switch_overhead_us);
-  if (rc != GCAPS_OK) return rc;
+  return gcaps_rta_batch_host_multi(ts, n_tasksets, &policy, 1, timeslice_us, ctx_switch_overhead_us,
+                                    &out_wcrt, &out_sched);
+}
+
+int gcaps_rta_batch_host_multi(const gcaps_tasksets_t *ts, int64_t n_tasksets, const int *policies,
+                               int n_policies, int64_t timeslice_us, int64_t ctx_switch_overhead_us,
+                               int64_t *const *out_wcrt, uint8_t *const *out_sched) {
+  if (!policies || n_policies < 1 || n_policies > kMaxHostPolicies || !out_wcrt || !out_sched)
+    return GCAPS_ERR_INVALID_ARG;
+  int rc = GCAPS_OK;
+  for (int q = 0; q < n_policies; ++q) {
+    rc = check_args(ts, n_tasksets, policies[q], timeslice_us, ctx_switch_overhead_us);
+    if (rc != GCAPS_OK) return rc;
+  }
   if (n_tasksets == 0) return GCAPS_OK;
-  if (!out_sched || (ts->n_tasks > 0 && !out_wcrt)) return GCAPS_ERR_INVALID_ARG;
+  for (int q = 0; q < n_policies; ++q)
+    if (!out_sched[q] || (ts->n_tasks > 0 && !out_wcrt[q])) return GCAPS_ERR_INVALID_ARG;
   DeviceInfo di;
   rc = device_info(&di);
   if (rc != GCAPS_OK) return rc;
@@ -1460,8 +1481,8 @@ int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int pol
       t1 += 1;
     }
     if (t1 > t && host_range_is_canonical(ts, k0, k1)) {
-      rc = host_chunk(ts, t, t1, policy, timeslice_us, ctx_switch_overhead_us, out_wcrt, out_sched,
-                      slot, di.sm_count);
+      rc = host_chunk(ts, t, t1, policies, n_policies, timeslice_us, ctx_switch_overhead_us,
+                      out_wcrt, out_sched, slot, di.sm_count);
       if (rc != GCAPS_OK) return rc;
       slot ^= 1;
       t = t1;
@@ -1473,13 +1494,15 @@ int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int pol
     for (; t < stop; ++t) {
       const int64_t a = ts->task_off[t], b = ts->task_off[t + 1];
       if (a < 0 || b < a || b > ts->n_tasks || b - a > GCAPS_RTA_MAX_TASKS) {
-        out_sched[t] = GCAPS_SCHED_INVALID;
+        for (int q = 0; q < n_policies; ++q) out_sched[q][t] = GCAPS_SCHED_INVALID;
       } else if (!host_range_is_canonical(ts, a, b)) {
-        out_sched[t] = GCAPS_SCHED_INVALID;
-        for (int64_t k = a; k < b; ++k) out_wcrt[k] = GCAPS_WCRT_INVALID;
+        for (int q = 0; q < n_policies; ++q) {
+          out_sched[q][t] = GCAPS_SCHED_INVALID;
+          for (int64_t k = a; k < b; ++k) out_wcrt[q][k] = GCAPS_WCRT_INVALID;
+        }
       } else {
-        rc = host_chunk(ts, t, t + 1, policy, timeslice_us, ctx_switch_overhead_us, out_wcrt,
-                        out_sched, slot, di.sm_count);
+        rc = host_chunk(ts, t, t + 1, policies, n_policies, timeslice_us, ctx_switch_overhead_us,
+                        out_wcrt, out_sched, slot, di.sm_count);
         if (rc != GCAPS_OK) return rc;
         slot ^= 1;
       }

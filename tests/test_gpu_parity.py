@@ -304,6 +304,18 @@ def test_host_buffer_entry_point():
     w_ref, s_ref, _ = rta.analyse(broken, 0, 512, 25)
     w, s = binding.rta_batch_host(broken.arrays(), 0, 512, 25)
     assert (s == s_ref).all() and (w == w_ref).all()
+    # several analyses of one copy of the inputs
+    pols = [0, 1, BUSY, 1 | BUSY | LITERAL]
+    ws, ss = binding.rta_batch_host_multi(b.arrays(), pols, 1024, 50)
+    for q, policy in enumerate(pols):
+        w_ref, s_ref, _ = rta.analyse(b, policy, 1024, 50)
+        assert (ss[q] == s_ref).all() and (ws[q] == w_ref).all(), policy
+    ws, ss = binding.rta_batch_host_multi(broken.arrays(), [0, 1], 512, 25)
+    for q, policy in enumerate([0, 1]):
+        w_ref, s_ref, _ = rta.analyse(broken, policy, 512, 25)
+        assert (ss[q] == s_ref).all() and (ws[q] == w_ref).all(), policy
+    with pytest.raises(binding.GcapsError):
+        binding.rta_batch_host_multi(small.arrays(), [0] * 9, 512, 25)
     binding.release_host()
 
 
