@@ -31,7 +31,8 @@ FALLBACK_HBM_GBS = 6650.0
 # plain-ALU peak of one B200: 148 SMs x 128 INT32 lanes x 1.965 GHz (integer lane-operations/s)
 ALU_PEAK_LANEOPS = 148 * 128 * 1.965e9
 K_TERM, K_SETUP = 6, 16   # algorithmic integer lane-operations per interference term / per task
-# kernels launched by one gcaps_rta_batch call: 3 plan kernels + one analysis kernel per size bin
+# kernels launched by one gcaps_rta_batch call: 3 plan kernels, one analysis kernel for the bins
+# of up to 32 tasks and one each for the 64-, 96-, 128-, 192- and 256-task bins
 LAUNCHES_PER_CALL = 9
 # DRAM bytes (read + write) per taskset of the analysis kernel on the 'large' workload, from the
 # ncu capture summarised in profiles/rta_kernel_large_131072_full.md (131,072 tasksets; traffic

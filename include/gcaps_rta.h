@@ -197,7 +197,7 @@ int gcaps_rta_batch_host_multi(const gcaps_tasksets_t *ts, int64_t n_tasksets, c
  *     stream, or otherwise ordered, are safe.
  */
 #define GCAPS_RTA_STATIC_MAX_TASKSETS 65536
-#define GCAPS_RTA_STATIC_SCRATCH_BYTES (256 + 2048 + 4 * GCAPS_RTA_STATIC_MAX_TASKSETS)
+#define GCAPS_RTA_STATIC_SCRATCH_BYTES (256 + 3072 + 4 * GCAPS_RTA_STATIC_MAX_TASKSETS)
 int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
                            int64_t timeslice_us, int64_t ctx_switch_overhead_us,
                            int64_t *out_wcrt, uint8_t *out_sched, void *stream);

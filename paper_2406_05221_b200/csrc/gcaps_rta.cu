@@ -35,9 +35,10 @@ namespace {
 typedef unsigned long long u64;
 typedef long long i64;
 
-constexpr int kNumBins = 6;
+constexpr int kNumBins = 9;
+constexpr int kBinStride = 12;  // counters per plan block and per header array
 typedef unsigned int u32;
-// size bins: at most 32, 64, 96, 128, 192, 256 tasks = 1, 2, 3, 4, 6, 8 tasks per lane
+// size bins: at most 8, 16, 24, 32, 64, 96, 128, 192, 256 tasks
 constexpr u32 kFastLimit = 1u << 26;  // fast path: every time of the taskset is below this
 constexpr u32 kFastClamp = 1u << 26;  // ... so a sum clamped here still exceeds every deadline
 constexpr int kBlockThreads = 128;
@@ -45,12 +46,11 @@ constexpr int kPlanItems = 1024;  // tasksets per plan block
 constexpr u64 kClamp = 1ull << 50;  // any quantity >= 2^50 exceeds every deadline (<= 2^40)
 
 struct PlanHeader {
-  unsigned int bin_start[8];
-  unsigned int bin_count[8];
-  unsigned int next[8];  // work counters of the analysis launches
-  unsigned int pad[8];
+  unsigned int bin_start[kBinStride];
+  unsigned int bin_count[kBinStride];
+  unsigned int next[kBinStride];  // work counters of the analysis launches
 };
-static_assert(sizeof(PlanHeader) == 128, "header layout");
+static_assert(sizeof(PlanHeader) <= 256, "header layout");
 
 struct KParams {
   const i64 *task_off, *period, *deadline, *priority, *core;
@@ -66,17 +66,20 @@ struct KParams {
   i64 *out_wcrt;
   uint8_t *out_sched;
   PlanHeader *hdr;
-  unsigned int *block_cnt;  // [plan blocks][8]
+  unsigned int *block_cnt;  // [plan blocks][kBinStride]
   unsigned int *perm;       // [n_tasksets]
 };
 
 __device__ __forceinline__ int size_bin(i64 n) {
-  if (n <= 32) return 0;  // also negative / broken ranges: rejected by the analysis kernel
-  if (n <= 64) return 1;
-  if (n <= 96) return 2;
-  if (n <= 128) return 3;
-  if (n <= 192) return 4;
-  if (n <= GCAPS_RTA_MAX_TASKS) return 5;
+  if (n <= 8) return 0;  // also negative / broken ranges: rejected by the analysis kernel
+  if (n <= 16) return 1;
+  if (n <= 24) return 2;
+  if (n <= 32) return 3;
+  if (n <= 64) return 4;
+  if (n <= 96) return 5;
+  if (n <= 128) return 6;
+  if (n <= 192) return 7;
+  if (n <= GCAPS_RTA_MAX_TASKS) return 8;
   return 0;
 }
 
@@ -84,8 +87,8 @@ __device__ __forceinline__ int size_bin(i64 n) {
 // plan: counting sort of taskset indices by size bin (histogram per block, scan, scatter)
 // ---------------------------------------------------------------------------------------------
 __global__ void plan_count_kernel(KParams p) {
-  __shared__ unsigned int cnt[8];
-  if (threadIdx.x < 8) cnt[threadIdx.x] = 0;
+  __shared__ unsigned int cnt[kBinStride];
+  if (threadIdx.x < kBinStride) cnt[threadIdx.x] = 0;
   __syncthreads();
   i64 t0 = (i64)blockIdx.x * kPlanItems;
   for (int k = threadIdx.x; k < kPlanItems; k += blockDim.x) {
@@ -93,58 +96,48 @@ __global__ void plan_count_kernel(KParams p) {
     if (t < p.n_tasksets) atomicAdd(&cnt[size_bin(p.task_off[t + 1] - p.task_off[t])], 1u);
   }
   __syncthreads();
-  if (threadIdx.x < 8) p.block_cnt[(size_t)blockIdx.x * 8 + threadIdx.x] = cnt[threadIdx.x];
+  if (threadIdx.x < kBinStride)
+    p.block_cnt[(size_t)blockIdx.x * kBinStride + threadIdx.x] = cnt[threadIdx.x];
 }
 
-// One block.  Turns per-block counts into per-block write cursors and fills the header.
+// One block, one warp per bin.  Turns per-block counts into per-block write cursors and fills the
+// header.
 __global__ void plan_scan_kernel(KParams p, unsigned int n_blocks) {
-  __shared__ unsigned int warp_tot[32];
-  __shared__ unsigned int carry;
-  __shared__ unsigned int bin_total[8];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-  for (int b = 0; b < kNumBins; ++b) {
-    if (threadIdx.x == 0) carry = 0;
-    __syncthreads();
-    for (unsigned int base = 0; base < n_blocks; base += blockDim.x) {
-      unsigned int i = base + threadIdx.x;
-      unsigned int v = i < n_blocks ? p.block_cnt[(size_t)i * 8 + b] : 0u;
+  __shared__ unsigned int bin_total[kBinStride];
+  const int lane = threadIdx.x & 31, b = threadIdx.x >> 5;
+  if (b < kNumBins) {
+    unsigned int carry = 0;
+    for (unsigned int base = 0; base < n_blocks; base += 32) {
+      const unsigned int i = base + lane;
+      const unsigned int v = i < n_blocks ? p.block_cnt[(size_t)i * kBinStride + b] : 0u;
       unsigned int x = v;
+#pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
-        unsigned int y = __shfl_up_sync(0xffffffffu, x, d);
+        const unsigned int y = __shfl_up_sync(0xffffffffu, x, d);
         if (lane >= d) x += y;
       }
-      if (lane == 31) warp_tot[warp] = x;
-      __syncthreads();
-      unsigned int before = 0;
-      for (int w = 0; w < warp; ++w) before += warp_tot[w];
-      unsigned int excl = carry + before + x - v;
-      if (i < n_blocks) p.block_cnt[(size_t)i * 8 + b] = excl;  // cursor relative to the bin
-      __syncthreads();
-      if (threadIdx.x == blockDim.x - 1) {
-        unsigned int tot = 0;
-        for (int w = 0; w < n_warps; ++w) tot += warp_tot[w];
-        carry += tot;
-      }
-      __syncthreads();
+      if (i < n_blocks) p.block_cnt[(size_t)i * kBinStride + b] = carry + x - v;  // cursor within the bin
+      carry += __shfl_sync(0xffffffffu, x, 31);
     }
-    if (threadIdx.x == 0) bin_total[b] = carry;
-    __syncthreads();
+    if (lane == 0) bin_total[b] = carry;
   }
+  __syncthreads();
   if (threadIdx.x == 0) {
     unsigned int s = 0;
-    for (int b = 0; b < 8; ++b) {
-      unsigned int c = b < kNumBins ? bin_total[b] : 0u;
-      p.hdr->bin_start[b] = s;
-      p.hdr->bin_count[b] = c;
-      p.hdr->next[b] = 0;
+    for (int k = 0; k < kBinStride; ++k) {
+      const unsigned int c = k < kNumBins ? bin_total[k] : 0u;
+      p.hdr->bin_start[k] = s;
+      p.hdr->bin_count[k] = c;
+      p.hdr->next[k] = 0;
       s += c;
     }
   }
 }
 
 __global__ void plan_scatter_kernel(KParams p) {
-  __shared__ unsigned int cursor[8];
-  if (threadIdx.x < 8) cursor[threadIdx.x] = p.block_cnt[(size_t)blockIdx.x * 8 + threadIdx.x];
+  __shared__ unsigned int cursor[kBinStride];
+  if (threadIdx.x < kBinStride)
+    cursor[threadIdx.x] = p.block_cnt[(size_t)blockIdx.x * kBinStride + threadIdx.x];
   __syncthreads();
   i64 t0 = (i64)blockIdx.x * kPlanItems;
   for (int k = threadIdx.x; k < kPlanItems; k += blockDim.x) {
@@ -480,75 +473,77 @@ __device__ __forceinline__ bool slice_is_inside(i64 first, int N, int par, i64 t
   return (par == 0 || first >= 1) && ((((N + par) & 1) == 0) || first + N < total);
 }
 
-template <int SLOTS>
+template <int LPT, int SLOTS>
 struct FastLayout {
-  static constexpr int MAXN = 32 * SLOTS;
-  // a prefix array takes slices of up to CAP-1 elements and is written 128 words at a time
-  static constexpr int CAP = (6 * MAXN + 127) / 128 * 128;
+  static constexpr int MAXN = LPT * SLOTS;
+  static constexpr int kStep = 4 * LPT;  // elements one prefix step of the group covers
+  // a prefix array takes slices of up to CAP-1 elements and is written kStep words at a time
+  static constexpr int CAP = (6 * MAXN + kStep - 1) / kStep * kStep;
   static constexpr int kInfo = 0;  // uint4 per rank: deadline, core, base, position | GPU flag
   static constexpr int kQ0 = 4 * MAXN + 4;
   static constexpr int kQ1 = kQ0 + CAP + 4;
   static constexpr int kFastWords = kQ1 + CAP;
   static constexpr int kExactWords = (17 * MAXN + 3) / 4 * 4;  // the exact path: 66 B per task
   static constexpr int kWords = kFastWords > kExactWords ? kFastWords : kExactWords;
-  static_assert(kWords % 4 == 0 && CAP % 128 == 0 && 4 * MAXN <= CAP, "16-byte aligned rows");
+  static_assert(kWords % 4 == 0 && CAP % kStep == 0 && 4 * MAXN <= CAP, "16-byte aligned rows");
 };
 
-// One 128*NB-element step of the running sums of up to two arrays that share their offsets.
-template <int NB, bool TWO>
+// One step (NB blocks of 4*LPT elements) of the running sums of up to two arrays that share their
+// offsets, by a group of LPT lanes (`gmask`).
+template <int LPT, int NB, bool TWO>
 __device__ __forceinline__ void prefix_step(const i64 *__restrict__ X0, const i64 *__restrict__ X1,
                                             int e0, int N, int par0, int par1, bool inside,
                                             const i64 *lo0, const i64 *hi0, const i64 *lo1,
                                             const i64 *hi1, u32 *Q0, u32 *Q1, u32 &carry0,
-                                            u32 &carry1, u32 &bad, int lane) {
+                                            u32 &carry1, u32 &bad, int lane, unsigned int gmask) {
   Quad q0[NB], q1[NB];
   u32 x0[NB][4], x1[NB][4], i0[NB], i1[NB];
   if (inside) {
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      load_quad_inside(X0, e0 + 128 * b + 4 * lane - par0, N, q0[b]);
-      if (TWO) load_quad_inside(X1, e0 + 128 * b + 4 * lane - par1, N, q1[b]);
+      load_quad_inside(X0, e0 + 4 * LPT * b + 4 * lane - par0, N, q0[b]);
+      if (TWO) load_quad_inside(X1, e0 + 4 * LPT * b + 4 * lane - par1, N, q1[b]);
     }
   } else {
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      q0[b] = load_quad_edge(X0, e0 + 128 * b + 4 * lane - par0, N, lo0, hi0);
-      if (TWO) q1[b] = load_quad_edge(X1, e0 + 128 * b + 4 * lane - par1, N, lo1, hi1);
+      q0[b] = load_quad_edge(X0, e0 + 4 * LPT * b + 4 * lane - par0, N, lo0, hi0);
+      if (TWO) q1[b] = load_quad_edge(X1, e0 + 4 * LPT * b + 4 * lane - par1, N, lo1, hi1);
     }
   }
 #pragma unroll
   for (int b = 0; b < NB; ++b) {
-    narrow_quad(q0[b], e0 + 128 * b + 4 * lane - par0, N, x0[b], bad);
+    narrow_quad(q0[b], e0 + 4 * LPT * b + 4 * lane - par0, N, x0[b], bad);
     i0[b] = x0[b][3];
     if (TWO) {
-      narrow_quad(q1[b], e0 + 128 * b + 4 * lane - par1, N, x1[b], bad);
+      narrow_quad(q1[b], e0 + 4 * LPT * b + 4 * lane - par1, N, x1[b], bad);
       i1[b] = x1[b][3];
     }
   }
 #pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {  // the warp scans of all blocks side by side
+  for (int d = 1; d < LPT; d <<= 1) {  // the warp scans of all blocks side by side
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      const u32 y0 = __shfl_up_sync(kFull, i0[b], d);
+      const u32 y0 = __shfl_up_sync(gmask, i0[b], d, LPT);
       if (lane >= d) i0[b] += y0;
       if (TWO) {
-        const u32 y1 = __shfl_up_sync(kFull, i1[b], d);
+        const u32 y1 = __shfl_up_sync(gmask, i1[b], d, LPT);
         if (lane >= d) i1[b] += y1;
       }
     }
   }
 #pragma unroll
   for (int b = 0; b < NB; ++b) {
-    if (e0 + 128 * b < N + 1) {
+    if (e0 + 4 * LPT * b < N + 1) {
       const u32 b0 = i0[b] - x0[b][3] + carry0;
-      *reinterpret_cast<uint4 *>(Q0 + e0 + 128 * b + 4 * lane) =
+      *reinterpret_cast<uint4 *>(Q0 + e0 + 4 * LPT * b + 4 * lane) =
           make_uint4(x0[b][0] + b0, x0[b][1] + b0, x0[b][2] + b0, x0[b][3] + b0);
-      carry0 += __shfl_sync(kFull, i0[b], 31);
+      carry0 += __shfl_sync(gmask, i0[b], LPT - 1, LPT);
       if (TWO) {
         const u32 b1 = i1[b] - x1[b][3] + carry1;
-        *reinterpret_cast<uint4 *>(Q1 + e0 + 128 * b + 4 * lane) =
+        *reinterpret_cast<uint4 *>(Q1 + e0 + 4 * LPT * b + 4 * lane) =
             make_uint4(x1[b][0] + b1, x1[b][1] + b1, x1[b][2] + b1, x1[b][3] + b1);
-        carry1 += __shfl_sync(kFull, i1[b], 31);
+        carry1 += __shfl_sync(gmask, i1[b], LPT - 1, LPT);
       }
     }
   }
@@ -558,15 +553,18 @@ __device__ __forceinline__ void prefix_step(const i64 *__restrict__ X0, const i6
 // Returns false, having written nothing, if the taskset is not eligible for 32-bit arithmetic
 // (or is invalid): the caller then runs the exact 64-bit path, which also does the validation.
 //
-// Until the per-task sums are known lane l holds the tasks at positions l, l+32, ... ("slots").
+// A group of LPT lanes (8, 16 or a whole warp) works on one taskset.  Until the per-task sums are
+// known lane l of the group holds the tasks at positions l, l+LPT, ... ("slots").
 // Then every task's values move through shared memory to the lane that owns its rank, so that the
-// interferers of the task of rank `pos` sit in lanes (pos-1) % 32 downwards of slots up to
-// (pos-1) / 32 and higher slots can be skipped.
-template <int SLOTS, int MODE>
-__device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane) {
-  typedef FastLayout<SLOTS> Lay;
+// interferers of the task of rank `pos` sit in lanes (pos-1) % LPT downwards of slots up to
+// (pos-1) / LPT and higher slots can be skipped.
+template <int LPT, int SLOTS, int MODE>
+__device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane,
+                                             unsigned int gmask) {
+  typedef FastLayout<LPT, SLOTS> Lay;
+  constexpr int kLog = LPT == 32 ? 5 : LPT == 16 ? 4 : 3;  // log2 of the lanes per taskset
   constexpr int MAXN = Lay::MAXN, CAP = Lay::CAP;
-  constexpr int BC = SLOTS <= 2 ? SLOTS : 2;  // 128-element steps whose loads are issued together
+  constexpr int BC = SLOTS <= 2 ? SLOTS : 2;  // prefix blocks whose loads are issued together
   constexpr int BG = 1;
   constexpr bool kGcaps = MODE < 2;
   const bool literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
@@ -583,13 +581,13 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     i64 t64[SLOTS], d64[SLOTS], pr[SLOTS], c64[SLOTS], co[SLOTS], go[SLOTS];
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {  // all loads of the taskset's per-task arrays in flight
-      const i64 k = a + (lane + 32 * s < n ? lane + 32 * s : 0);
+      const i64 k = a + (lane + LPT * s < n ? lane + LPT * s : 0);
       t64[s] = p.period[k], d64[s] = p.deadline[k], pr[s] = p.priority[k], c64[s] = p.core[k];
       co[s] = p.cseg_off[k], go[s] = p.gseg_off[k];
     }
     const i64 cend = p.cseg_off[a + n] - p.cseg_base, gend = p.gseg_off[a + n] - p.gseg_base;
-    cfirst = __shfl_sync(kFull, co[0], 0) - p.cseg_base;
-    gfirst = __shfl_sync(kFull, go[0], 0) - p.gseg_base;
+    cfirst = __shfl_sync(gmask, co[0], 0, LPT) - p.cseg_base;
+    gfirst = __shfl_sync(gmask, go[0], 0, LPT) - p.gseg_base;
     const i64 Nc64 = cend - cfirst, Ng64 = gend - gfirst;
     if (cfirst < 0 || Nc64 < 0 || cend > p.n_csegs || Nc64 >= CAP || gfirst < 0 || Ng64 < 0 ||
         gend > p.n_gsegs || Ng64 >= CAP)
@@ -600,7 +598,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     int prio[SLOTS];
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
-      const bool v = lane + 32 * s < n;
+      const bool v = lane + LPT * s < n;
       const i64 rc = co[s] - p.cseg_base - cfirst, rg = go[s] - p.gseg_base - gfirst;
       const u32 h = (u32)((u64)t64[s] >> 32) | (u32)((u64)d64[s] >> 32) | (u32)((u64)c64[s] >> 32) |
                     (u32)((u64)rc >> 32) | (u32)((u64)rg >> 32) |
@@ -616,37 +614,37 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       ok &= T[s] - 2u < kFastLimit - 2u && (!v || (D[s] - 1u < T[s] && (int)core[s] >= 0)) &&
             (u32)c0[s] <= (u32)Nc && (u32)g0[s] <= (u32)Ng;
     }
-    if (__any_sync(kFull, high != 0 || !ok)) return false;  // (a wide priority also lands here)
+    if (__any_sync(gmask, high != 0 || !ok)) return false;  // (a wide priority also lands here)
     // order: rank by (priority desc, position asc)
     int m = prio[0];
 #pragma unroll
     for (int s = 1; s < SLOTS; ++s) m = prio[s] > m ? prio[s] : m;
-    const int pmax = __reduce_max_sync(kFull, m);
+    const int pmax = __reduce_max_sync(gmask, m);
     bool dense = true;  // distinct priorities max-n+1 .. max: the rank is max - priority
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
       const u32 r = (u32)pmax - (u32)prio[s];
-      const bool v = lane + 32 * s < n;
+      const bool v = lane + LPT * s < n;
       dense &= !v || r < (u32)n;
       rank[s] = v ? (int)r : MAXN;
     }
-    dense = __all_sync(kFull, dense);
+    dense = __all_sync(gmask, dense);
     if (dense) {
 #pragma unroll
       for (int s = 0; s < SLOTS; ++s)
-        if (lane + 32 * s < n) Q0[rank[s]] = (u32)(lane + 32 * s);
-      __syncwarp();
+        if (lane + LPT * s < n) Q0[rank[s]] = (u32)(lane + LPT * s);
+      __syncwarp(gmask);
       bool uniq = true;
 #pragma unroll
       for (int s = 0; s < SLOTS; ++s)
-        if (lane + 32 * s < n) uniq &= Q0[rank[s]] == (u32)(lane + 32 * s);
-      dense = __all_sync(kFull, uniq);
-      __syncwarp();
+        if (lane + LPT * s < n) uniq &= Q0[rank[s]] == (u32)(lane + LPT * s);
+      dense = __all_sync(gmask, uniq);
+      __syncwarp(gmask);
     }
     if (!dense) {  // any priorities: count the tasks that come before
 #pragma unroll
       for (int s = 0; s < SLOTS; ++s) {
-        const int i = lane + 32 * s;
+        const int i = lane + LPT * s;
         int r = 0;
         for (int q = 0; q < n; ++q) {
           const int pq = (int)p.priority[a + q];
@@ -658,21 +656,21 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     // what every lane must know about the task of a given rank (base and GPU flag follow)
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s)
-      if (lane + 32 * s < n)
+      if (lane + LPT * s < n)
         *reinterpret_cast<uint2 *>(&info[rank[s]]) = make_uint2(D[s], core[s]);
   }
   // end offsets: the next task's start (positions beyond n hold the total)
   int c1[SLOTS], g1[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    const int cn = __shfl_down_sync(kFull, c0[s], 1), gn = __shfl_down_sync(kFull, g0[s], 1);
-    const int ch = __shfl_sync(kFull, s + 1 < SLOTS ? c0[s + 1 < SLOTS ? s + 1 : s] : Nc, 0);
-    const int gh = __shfl_sync(kFull, s + 1 < SLOTS ? g0[s + 1 < SLOTS ? s + 1 : s] : Ng, 0);
-    c1[s] = lane == 31 ? ch : cn;
-    g1[s] = lane == 31 ? gh : gn;
+    const int cn = __shfl_down_sync(gmask, c0[s], 1, LPT), gn = __shfl_down_sync(gmask, g0[s], 1, LPT);
+    const int ch = __shfl_sync(gmask, s + 1 < SLOTS ? c0[s + 1 < SLOTS ? s + 1 : s] : Nc, 0, LPT);
+    const int gh = __shfl_sync(gmask, s + 1 < SLOTS ? g0[s + 1 < SLOTS ? s + 1 : s] : Ng, 0, LPT);
+    c1[s] = lane == LPT - 1 ? ch : cn;
+    g1[s] = lane == LPT - 1 ? gh : gn;
     ok &= (u32)(c1[s] - c0[s]) < 64u && (u32)(g1[s] - g0[s]) < 64u;
   }
-  if (!__all_sync(kFull, ok)) return false;
+  if (!__all_sync(gmask, ok)) return false;
 
   // ---- aggregate: running sums of the segment arrays; per-task sums are differences --------
   u32 A[SLOTS], Ge[SLOTS], S[SLOTS];  // C+G^m, G^e, and 2*eps*eta (GCAPS) or (L+theta)*slices (RR)
@@ -685,23 +683,23 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   {  // CPU segments -> Q0
     const bool inside = slice_is_inside(cfirst, Nc, parc, p.n_csegs);
     u32 carry = 0, unused = 0;
-    for (int e0 = 0; e0 < Nc + parc; e0 += 128 * BC)
-      prefix_step<BC, false>(Xc, Xc, e0, Nc, parc, parc, inside, p.cseg_wcet, p.cseg_wcet + p.n_csegs,
-                             p.cseg_wcet, p.cseg_wcet, Q0, Q0, carry, unused, bad, lane);
+    for (int e0 = 0; e0 < Nc + parc; e0 += Lay::kStep * BC)
+      prefix_step<LPT, BC, false>(Xc, Xc, e0, Nc, parc, parc, inside, p.cseg_wcet, p.cseg_wcet + p.n_csegs,
+                             p.cseg_wcet, p.cseg_wcet, Q0, Q0, carry, unused, bad, lane, gmask);
   }
-  __syncwarp();
+  __syncwarp(gmask);
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) A[s] = Q0[c1[s] - 1 + parc] - Q0[c0[s] - 1 + parc];
-  __syncwarp();
+  __syncwarp(gmask);
   {  // G^m -> Q0, G^e -> Q1
     const bool inside = slice_is_inside(gfirst, Ng, parm, p.n_gsegs) &&
                         slice_is_inside(gfirst, Ng, pare, p.n_gsegs);
     u32 cm = 0, ce = 0;
-    for (int e0 = 0; e0 < Ng + 1; e0 += 128 * BG)
-      prefix_step<BG, true>(Xm, Xe, e0, Ng, parm, pare, inside, p.gseg_misc, p.gseg_misc + p.n_gsegs,
-                            p.gseg_exec, p.gseg_exec + p.n_gsegs, Q0, Q1, cm, ce, bad, lane);
+    for (int e0 = 0; e0 < Ng + 1; e0 += Lay::kStep * BG)
+      prefix_step<LPT, BG, true>(Xm, Xe, e0, Ng, parm, pare, inside, p.gseg_misc, p.gseg_misc + p.n_gsegs,
+                            p.gseg_exec, p.gseg_exec + p.n_gsegs, Q0, Q1, cm, ce, bad, lane, gmask);
   }
-  __syncwarp();
+  __syncwarp(gmask);
   u32 eta[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
@@ -712,17 +710,17 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     A[s] += Gm;
     bad |= A[s] >> 26;
   }
-  __syncwarp();
+  __syncwarp(gmask);
   if (!kGcaps) {  // Eq. 3: slices of every pure GPU part, summed per task (values already checked)
     const bool inside = slice_is_inside(gfirst, Ng, pare, p.n_gsegs);
     u32 carry = 0;
-    for (int e0 = 0; e0 < Ng + 1; e0 += 128 * BG) {
+    for (int e0 = 0; e0 < Ng + 1; e0 += Lay::kStep * BG) {
       Quad qe[BG];
       u32 x[BG][4], incl[BG];
 #pragma unroll
       for (int b = 0; b < BG; ++b) {
-        if (inside) load_quad_inside(Xe, e0 + 128 * b + 4 * lane - pare, Ng, qe[b]);
-        else qe[b] = load_quad_edge(Xe, e0 + 128 * b + 4 * lane - pare, Ng, p.gseg_exec, p.gseg_exec + p.n_gsegs);
+        if (inside) load_quad_inside(Xe, e0 + 4 * LPT * b + 4 * lane - pare, Ng, qe[b]);
+        else qe[b] = load_quad_edge(Xe, e0 + 4 * LPT * b + 4 * lane - pare, Ng, p.gseg_exec, p.gseg_exec + p.n_gsegs);
       }
 #pragma unroll
       for (int b = 0; b < BG; ++b) {
@@ -739,29 +737,29 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
         incl[b] = x[b][3];
       }
 #pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
+      for (int d = 1; d < LPT; d <<= 1) {
 #pragma unroll
         for (int b = 0; b < BG; ++b) {
-          const u32 y = __shfl_up_sync(kFull, incl[b], d);
+          const u32 y = __shfl_up_sync(gmask, incl[b], d, LPT);
           if (lane >= d) incl[b] += y;
         }
       }
 #pragma unroll
       for (int b = 0; b < BG; ++b) {
-        if (e0 + 128 * b < Ng + 1) {
+        if (e0 + 4 * LPT * b < Ng + 1) {
           const u32 before = incl[b] - x[b][3] + carry;
-          *reinterpret_cast<uint4 *>(Q0 + e0 + 128 * b + 4 * lane) =
+          *reinterpret_cast<uint4 *>(Q0 + e0 + 4 * LPT * b + 4 * lane) =
               make_uint4(x[b][0] + before, x[b][1] + before, x[b][2] + before, x[b][3] + before);
-          carry += __shfl_sync(kFull, incl[b], 31);
+          carry += __shfl_sync(gmask, incl[b], LPT - 1, LPT);
         }
       }
     }
-    __syncwarp();
+    __syncwarp(gmask);
   }
   // ---- constants of Eq. 1 that do not depend on R ------------------------------------------
   int n_gpu = 0;  // N_g
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(kFull, eta[s] > 0));
+  for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(gmask, eta[s] > 0));
   const u32 ovh = (u32)p.ovh;  // the fast path is only entered with eps, theta < 2^20
   u32 base[SLOTS];
 #pragma unroll
@@ -781,24 +779,24 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     }
     base[s] = base[s] > 2 * kFastClamp ? 2 * kFastClamp : base[s];
   }
-  if (__any_sync(kFull, bad != 0)) return false;
-  __syncwarp();
+  if (__any_sync(gmask, bad != 0)) return false;
+  __syncwarp(gmask);
   // ---- move every task to the lane that owns its rank -------------------------------------
   uint4 *xch = reinterpret_cast<uint4 *>(Q0);  // by rank: T, C+G^m, G^e, S  (Q0, Q1 are dead now)
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    if (lane + 32 * s < n) {
+    if (lane + LPT * s < n) {
       *(reinterpret_cast<uint2 *>(&info[rank[s]]) + 1) =
-          make_uint2(base[s], (u32)(lane + 32 * s) | (eta[s] > 0 ? 0x10000u : 0u));
+          make_uint2(base[s], (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u));
       xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], S[s]);
     }
   }
-  __syncwarp();
+  __syncwarp(gmask);
   u32 Tm1[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS], core[SLOTS];
   bool gpu[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    const int r = lane + 32 * s;
+    const int r = lane + LPT * s;
     const uint4 x = r < n ? xch[r] : make_uint4(2u, 0u, 0u, 0u);
     const uint4 f = r < n ? info[r] : make_uint4(0u, 0xffffffffu, 0u, 0u);
     Tm1[s] = x.x - 1, A[s] = x.y, Ge[s] = x.z, S[s] = x.w;
@@ -826,8 +824,8 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     const uint4 f = info[pos];
     const u32 Di = f.x, core_i = f.y, base_i = f.z;
     const bool gi = (f.w & 0x10000u) != 0;
-    const int smax = (pos - 1) >> 5;  // -1 for the first task: nothing interferes
-    if ((pos & 31) == 1) {            // the first task that looks at slot smax
+    const int smax = (pos - 1) >> kLog;  // -1 for the first task: nothing interferes
+    if ((pos & (LPT - 1)) == 1) {            // the first task that looks at slot smax
 #pragma unroll
       for (int s = 0; s < SLOTS; ++s)
         if (s == smax) make_reciprocal(Tm1[s] + 1, magic[s], shift[s]);
@@ -837,7 +835,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       int c = 0;
 #pragma unroll
       for (int s = 0; s < SLOTS; ++s)
-        if (s <= smax) c += __popc(__ballot_sync(kFull, lane + 32 * s < pos && core[s] == core_i && gpu[s]));
+        if (s <= smax) c += __popc(__ballot_sync(gmask, lane + LPT * s < pos && core[s] == core_i && gpu[s]));
       nu = (u32)(n_gpu - c + 1);
     }
     // the (J, W) pairs of this task's interferers; W = 0 where a pair does not apply
@@ -846,7 +844,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     for (int s = 0; s < SLOTS; ++s) {
       J1[s] = 0, W1[s] = 0, W2[s] = 0;
       if (s <= smax) {
-        const bool act = lane + 32 * s < pos;
+        const bool act = lane + LPT * s < pos;
         const bool same = core[s] == core_i;
         u32 w1, w2 = 0, j1;
         if (MODE == 0) {
@@ -891,7 +889,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
           }
         }
         const u32 part = acc > (u64)kFastClamp ? kFastClamp : (u32)acc;
-        next += __reduce_add_sync(kFull, part);
+        next += __reduce_add_sync(gmask, part);
       }
       if (next == R) break;
       R = next;
@@ -905,7 +903,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     // CPU-only task has no J^c unless the printed form of Lemma 7 is asked for)
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
-      if (lane + 32 * s == pos) {
+      if (lane + LPT * s == pos) {
         p.out_wcrt[a + pos_of[s]] = (i64)R;
         if (MODE == 0 ? gpu[s] : (MODE == 2 ? (gpu[s] || literal) : false)) Jc[s] = R - A[s] + Tm1[s];
         Jg[s] = R - Ge[s] + Tm1[s];
@@ -915,28 +913,29 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   // ---- write the sentinels of the tasks that did not converge ---------------------------------
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    const int r = lane + 32 * s;
+    const int r = lane + LPT * s;
     if (r < n && r >= n_done)
       p.out_wcrt[a + pos_of[s]] = r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED;
   }
   if (lane == 0) p.out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
-  __syncwarp();
+  __syncwarp(gmask);
   return true;
 }
-
-// What a warp knows in advance about one taskset of a chunk (kept in shared memory).
-struct Ahead {
-  i64 t, a;        // taskset index, first task
-  i64 c_lo, g_lo;  // first CPU segment, first GPU segment
-  int n, nc, ng;   // tasks, CPU segments, GPU segments (nc = ng = 0 unless the ranges are sound)
-  int fast;        // 1 if the task range is one the 32-bit path could take
-};
 
 __device__ __forceinline__ void prefetch_l2(const void *ptr) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
 }
-constexpr int kMaxChunk = 8;
-constexpr int kAheadWords = 2 * kMaxChunk * (int)(sizeof(Ahead) / sizeof(u32));  // two chunks
+
+// What a warp knows in advance about one taskset of a chunk (kept in shared memory).
+struct Ahead {
+  i64 a;           // first task
+  i64 c_lo, g_lo;  // first CPU segment, first GPU segment
+  u32 t;           // taskset index
+  u32 packed;      // tasks (bits 0-8) | CPU segments (9-19) | GPU segments (20-30) | fast (31)
+};
+static_assert(sizeof(Ahead) == 32, "two 16-byte rows");
+constexpr int kMaxAhead = 16;  // tasksets of one pull
+constexpr int kAheadWords = 2 * kMaxAhead * (int)(sizeof(Ahead) / sizeof(u32));  // two chunks
 
 // blocks per SM the register allocation aims at: more warps in flight matter more here than a
 // few spilled values, because every phase is a chain of dependent instructions and the loads of
@@ -945,88 +944,132 @@ __host__ __device__ constexpr int min_blocks(int slots) {
   return slots <= 3 ? 6 : slots == 4 ? 4 : slots == 6 ? 3 : 2;
 }
 
-// Persistent launch over one size bin: warps pull chunks of tasksets from the bin's counter; the
-// index and task range of the next chunk are fetched while the current one is analysed.
-template <int SLOTS, int MODE>
-__global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_kernel(KParams p, int bin) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  typedef FastLayout<SLOTS> Lay;
-  constexpr int MAXN = 32 * SLOTS;
-  constexpr int kWarpWords = Lay::kWords + kAheadWords;
+// One size bin, worked through by all warps of a persistent launch.  A warp is 32/LPT groups of
+// LPT lanes; every group analyses one taskset at a time.  Warps pull chunks of taskset indices
+// from the bin's counter; the index, task range and first segment offsets of the next chunk are
+// fetched while the current one is analysed.
+template <int LPT, int SLOTS, int MODE>
+__device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf, Ahead *ahead) {
+  typedef FastLayout<LPT, SLOTS> Lay;
+  constexpr int MAXN = LPT * SLOTS;
+  constexpr int G = 32 / LPT;  // groups per warp
   static_assert(sizeof(GroupSmem<MAXN>) <= sizeof(u32) * Lay::kWords, "exact path fits");
-  static_assert(kWarpWords % 4 == 0 && sizeof(Ahead) % 16 == 0, "alignment");
-  const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  u32 *buf = reinterpret_cast<u32 *>(smem_raw) + warp_in_block * kWarpWords;
-  Ahead *ahead = reinterpret_cast<Ahead *>(buf + Lay::kWords);  // [2][kMaxChunk]
+  const int lane32 = threadIdx.x & 31, group = lane32 / LPT, lane = lane32 % LPT;
+  const unsigned int gmask = LPT == 32 ? kFull : (((1u << LPT) - 1u) << (group * LPT));
+  u32 *buf = warp_buf + group * Lay::kWords;
   const unsigned int start = p.hdr->bin_start[bin], count = p.hdr->bin_count[bin];
+  if (count == 0) return;
   const bool fast_call = p.ovh < (1 << 20);  // keeps 2*eps*eta and (eta+1)*eps in 32 bits
-  // tasksets per pull: 8 when the bin is large, fewer when it would leave warps without work
-  const unsigned int n_warps = gridDim.x * (kBlockThreads / 32);
-  const int kChunk = count >= 32 * n_warps ? kMaxChunk : (count >= 8 * n_warps ? 4 : 1);
+  // tasksets per pull: up to 8 per group when the bin is large, fewer when that would leave warps
+  // without work
+  const unsigned int n_groups = gridDim.x * (kBlockThreads / 32) * G;
+  const int rounds = count >= 32 * n_groups ? (G == 1 ? 8 : kMaxAhead / G)
+                                            : (count >= 8 * n_groups ? 4 / (G > 2 ? 2 : 1) : 1);
+  const int chunk = rounds * G;  // <= kMaxAhead
 
-  // lanes 0..kChunk-1 each look up one taskset of a chunk and leave what they found in `slot`
+  // lanes 0..chunk-1 each look up one taskset of a chunk and leave what they found in `slot`
   auto look_up = [&](unsigned int first, Ahead *slot) {
-    if (lane < kChunk) {
+    if (lane32 < chunk) {
       Ahead me;
-      me.t = 0, me.a = 0, me.c_lo = me.g_lo = 0, me.n = me.nc = me.ng = 0, me.fast = 0;
-      if (first < count && first + lane < count) {
-        me.t = (i64)p.perm[start + first + lane];
+      me.a = 0, me.c_lo = me.g_lo = 0, me.t = 0, me.packed = 0;
+      if (first < count && first + lane32 < count) {
+        me.t = p.perm[start + first + lane32];
         me.a = p.task_off[me.t] - p.task_base;
-        const i64 b = p.task_off[me.t + 1] - p.task_base;
+        const i64 b = p.task_off[(i64)me.t + 1] - p.task_base;
         if (me.a >= 0 && b > me.a && b <= p.n_tasks && b - me.a <= MAXN) {
-          me.fast = 1, me.n = (int)(b - me.a);
+          u32 nc = 0, ng = 0;
           me.c_lo = p.cseg_off[me.a] - p.cseg_base, me.g_lo = p.gseg_off[me.a] - p.gseg_base;
           const i64 c_hi = p.cseg_off[b] - p.cseg_base, g_hi = p.gseg_off[b] - p.gseg_base;
           if (me.c_lo >= 0 && c_hi <= p.n_csegs && c_hi - me.c_lo < Lay::CAP && c_hi > me.c_lo)
-            me.nc = (int)(c_hi - me.c_lo);
+            nc = (u32)(c_hi - me.c_lo);
           if (me.g_lo >= 0 && g_hi <= p.n_gsegs && g_hi - me.g_lo < Lay::CAP && g_hi > me.g_lo)
-            me.ng = (int)(g_hi - me.g_lo);
+            ng = (u32)(g_hi - me.g_lo);
+          me.packed = (u32)(b - me.a) | (nc << 9) | (ng << 20) | 0x80000000u;
         }
       }
-      slot[lane] = me;
+      slot[lane32] = me;
     }
     __syncwarp();
   };
+  static_assert(MAXN <= 256 && Lay::CAP <= 2048, "fields of Ahead::packed");
 
   unsigned int first = 0;
-  if (lane == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
+  if (lane32 == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)chunk);
   first = __shfl_sync(kFull, first, 0);
   int which = 0;
   look_up(first, ahead);
   while (first < count) {
     unsigned int nfirst = 0;
-    if (lane == 0) nfirst = atomicAdd(&p.hdr->next[bin], (unsigned int)kChunk);
-    const Ahead *cur = ahead + which * kMaxChunk;
-    Ahead *nxt = ahead + (which ^ 1) * kMaxChunk;
-    const int in_chunk = count - first < (unsigned int)kChunk ? (int)(count - first) : kChunk;
-    for (int c = 0; c < in_chunk; ++c) {
-      if (c == 1 || in_chunk == 1) {  // the next chunk's index has arrived by now
+    if (lane32 == 0) nfirst = atomicAdd(&p.hdr->next[bin], (unsigned int)chunk);
+    const Ahead *cur = ahead + which * kMaxAhead;
+    Ahead *nxt = ahead + (which ^ 1) * kMaxAhead;
+    const int in_chunk = count - first < (unsigned int)chunk ? (int)(count - first) : chunk;
+    const int in_rounds = (in_chunk + G - 1) / G;
+    for (int c = 0; c < in_rounds; ++c) {
+      if (c == 1 || in_rounds == 1) {  // the next chunk's index has arrived by now
         nfirst = __shfl_sync(kFull, nfirst, 0);
         look_up(nfirst, nxt);
       }
-      const i64 t = cur[c].t, a = cur[c].a;
-      const int n = cur[c].n;
-      {  // the segment slices start their way into L2 now; the per-task loads follow at once, so
-         // that the running sums later wait for L2 rather than for DRAM (16 elements per line,
-         // only addresses inside the arrays)
-        const i64 c_lo = cur[c].c_lo, g_lo = cur[c].g_lo;
-        const int nc = cur[c].nc, ng = cur[c].ng;
-        for (int e = 16 * lane; e < nc; e += 16 * 32) prefetch_l2(p.cseg_wcet + c_lo + e);
-        for (int e = 16 * lane; e < ng; e += 16 * 32)
-          prefetch_l2(p.gseg_misc + g_lo + e), prefetch_l2(p.gseg_exec + g_lo + e);
-      }
-      bool done = false;
-      if (fast_call && cur[c].fast != 0) done = analyse_fast<SLOTS, MODE>(p, t, a, n, buf, lane);
-      __syncwarp();
-      if (!done) {
-        // the exact path reads task_off again and validates everything itself
-        analyse_taskset<32, MAXN>(p, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, kFull);
+      const int mine = c * G + group;
+      if (mine < in_chunk) {
+        const Ahead me = cur[mine];
+        const i64 t = (i64)me.t;
+        const int n = (int)(me.packed & 0x1ffu), nc = (int)((me.packed >> 9) & 0x7ffu);
+        const int ng = (int)((me.packed >> 20) & 0x7ffu);
+        // the segment slices start their way into L2 now; the per-task loads follow at once, so
+        // that the running sums later wait for L2 rather than for DRAM (16 elements per line,
+        // only addresses inside the arrays)
+        for (int e = 16 * lane; e < nc; e += 16 * LPT) prefetch_l2(p.cseg_wcet + me.c_lo + e);
+        for (int e = 16 * lane; e < ng; e += 16 * LPT)
+          prefetch_l2(p.gseg_misc + me.g_lo + e), prefetch_l2(p.gseg_exec + me.g_lo + e);
+        bool done = false;
+        if (fast_call && (me.packed >> 31) != 0)
+          done = analyse_fast<LPT, SLOTS, MODE>(p, t, me.a, n, buf, lane, gmask);
+        __syncwarp(gmask);
+        if (!done) {
+          // the exact path reads task_off again and validates everything itself
+          analyse_taskset<LPT, MAXN>(p, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, gmask);
+        }
       }
       __syncwarp();
     }
     first = nfirst;
     which ^= 1;
   }
+}
+
+// shared memory of one warp for the bins a kernel covers
+template <int LPT, int SLOTS>
+__host__ __device__ constexpr int bin_warp_words() {
+  return (32 / LPT) * FastLayout<LPT, SLOTS>::kWords;
+}
+__host__ __device__ constexpr int cmax(int a, int b) { return a > b ? a : b; }
+constexpr int kSmallWarpWords =
+    cmax(cmax(bin_warp_words<8, 1>(), bin_warp_words<8, 2>()),
+         cmax(bin_warp_words<8, 3>(), bin_warp_words<16, 2>())) + kAheadWords;
+
+// The bins of up to 32 tasks in one persistent launch, largest tasksets first: (lanes per
+// taskset, tasks per lane) = (16,2) (8,3) (8,2) (8,1) for at most 32, 24, 16, 8 tasks, i.e. two or
+// four tasksets per warp.
+template <int MODE>
+__global__ void __launch_bounds__(kBlockThreads, min_blocks(3)) rta_small_kernel(KParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
+  Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
+  run_bin<16, 2, MODE>(p, 3, warp_buf, ahead);
+  run_bin<8, 3, MODE>(p, 2, warp_buf, ahead);
+  run_bin<8, 2, MODE>(p, 1, warp_buf, ahead);
+  run_bin<8, 1, MODE>(p, 0, warp_buf, ahead);
+}
+
+// One bin of larger tasksets (a warp per taskset, 2, 3, 4, 6 or 8 tasks per lane) per launch.
+template <int SLOTS, int MODE>
+__global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kernel(KParams p, int bin) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
+  u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
+  Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
+  run_bin<32, SLOTS, MODE>(p, bin, warp_buf, ahead);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1152,42 +1195,51 @@ void fill_params(KParams *p, const gcaps_tasksets_t *ts, int64_t n_tasksets, int
   p->out_sched = out_sched;
 }
 
-template <int SLOTS, int MODE>
-cudaError_t launch_bin(const KParams &p, int bin, int sm_count, cudaStream_t st) {
-  constexpr int kWarps = kBlockThreads / 32;
-  const size_t smem = sizeof(u32) * (FastLayout<SLOTS>::kWords + kAheadWords) * kWarps;
-  static int blocks_per_sm[64] = {0};  // per device; 0 = not set up yet
+// Launches `kernel` (a persistent kernel of kBlockThreads threads needing `smem` bytes) with as
+// many blocks as the device keeps resident, but never more than the batch could feed.
+template <typename... Args>
+cudaError_t launch_persistent(void (*kernel)(Args...), int *blocks_per_sm, size_t smem, long long want,
+                              int sm_count, cudaStream_t st, Args... args) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   dev &= 63;
-  if (blocks_per_sm[dev] == 0) {
-    e = cudaFuncSetAttribute(rta_kernel<SLOTS, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem);
+  if (blocks_per_sm[dev] == 0) {  // first use on this device
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 1;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rta_kernel<SLOTS, MODE>,
-                                                      kBlockThreads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlockThreads, smem);
     if (e != cudaSuccess) return e;
     blocks_per_sm[dev] = per_sm < 1 ? 1 : per_sm;
   }
-  // never more warps than the bin could feed (the exact bin population lives on the device)
-  long long want = (p.n_tasksets + kWarps - 1) / kWarps;
   long long grid = (long long)sm_count * blocks_per_sm[dev];
   if (grid > want) grid = want;
   if (grid < 1) grid = 1;
-  rta_kernel<SLOTS, MODE><<<(unsigned int)grid, kBlockThreads, smem, st>>>(p, bin);
+  kernel<<<(unsigned int)grid, kBlockThreads, smem, st>>>(args...);
   return cudaGetLastError();
+}
+
+template <int SLOTS, int MODE>
+cudaError_t launch_big(const KParams &p, int bin, int sm_count, cudaStream_t st) {
+  constexpr int kWarps = kBlockThreads / 32;
+  static int blocks_per_sm[64] = {0};
+  const size_t smem = sizeof(u32) * (bin_warp_words<32, SLOTS>() + kAheadWords) * kWarps;
+  return launch_persistent(rta_big_kernel<SLOTS, MODE>, blocks_per_sm, smem,
+                           (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p, bin);
 }
 
 template <int MODE>
 cudaError_t launch_all_bins(const KParams &p, int sm_count, cudaStream_t st) {
-  cudaError_t e = launch_bin<1, MODE>(p, 0, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<2, MODE>(p, 1, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<3, MODE>(p, 2, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<4, MODE>(p, 3, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<6, MODE>(p, 4, sm_count, st);
-  if (e == cudaSuccess) e = launch_bin<8, MODE>(p, 5, sm_count, st);
+  constexpr int kWarps = kBlockThreads / 32;
+  static int blocks_per_sm[64] = {0};
+  const size_t smem = sizeof(u32) * kSmallWarpWords * kWarps;
+  cudaError_t e = launch_persistent(rta_small_kernel<MODE>, blocks_per_sm, smem,
+                                    (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p);
+  if (e == cudaSuccess) e = launch_big<2, MODE>(p, 4, sm_count, st);
+  if (e == cudaSuccess) e = launch_big<3, MODE>(p, 5, sm_count, st);
+  if (e == cudaSuccess) e = launch_big<4, MODE>(p, 6, sm_count, st);
+  if (e == cudaSuccess) e = launch_big<6, MODE>(p, 7, sm_count, st);
+  if (e == cudaSuccess) e = launch_big<8, MODE>(p, 8, sm_count, st);
   return e;
 }
 
@@ -1200,9 +1252,9 @@ int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_cou
   const size_t nb = plan_blocks(p.n_tasksets);
   p.hdr = (PlanHeader *)w;
   p.block_cnt = (unsigned int *)(w + 256);
-  p.perm = (unsigned int *)(w + 256 + align_up(nb * 8 * sizeof(unsigned int), 256));
+  p.perm = (unsigned int *)(w + 256 + align_up(nb * kBinStride * sizeof(unsigned int), 256));
   plan_count_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
-  plan_scan_kernel<<<1, 1024, 0, st>>>(p, (unsigned int)nb);
+  plan_scan_kernel<<<1, 32 * kNumBins, 0, st>>>(p, (unsigned int)nb);
   plan_scatter_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) {
@@ -1242,7 +1294,7 @@ extern "C" {
 size_t gcaps_rta_workspace_bytes(int64_t n_tasksets) {
   if (n_tasksets <= 0) return 0;
   const size_t nb = plan_blocks(n_tasksets);
-  return 256 + align_up(nb * 8 * sizeof(unsigned int), 256) +
+  return 256 + align_up(nb * kBinStride * sizeof(unsigned int), 256) +
          align_up((size_t)n_tasksets * sizeof(unsigned int), 256);
 }
 
