@@ -39,10 +39,10 @@ LAUNCHES_PER_CALL = 9
 # grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
 # the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "d4232a6525cddc1bcefe0fd16ad161304a6026db59e30f7dc84982e3f52c9270",
+    "source_sha256": "de335bca07754e68950253b73e2f4809f8d0244a3f70fc907aaed1ba700fbd57",
     "workload": "large",
-    "bytes_per_taskset": {"gcaps": (1247331000 + 82918656) / 131072.0,
-                          "rr": (1245120000 + 81220608) / 131072.0},
+    "bytes_per_taskset": {"gcaps": (1247450000 + 83256832) / 131072.0,
+                          "rr": (1245200000 + 81212160) / 131072.0},
 }
 
 
