@@ -22,7 +22,7 @@ def build(name: str, force: bool = False) -> str:
 
 
 def build_all(force: bool = False) -> None:
-    for name in ("rta_oracle", "des_sim"):
+    for name in ("rta_oracle", "gpu_prio_oracle", "des_sim"):
         build(name, force)
 
 

@@ -32,17 +32,19 @@ typedef struct {
 } job_shape_t;
 
 /*
- * n tasks; per task: T, prio (larger = higher, ties by index), core, offset, and the CSR segment
+ * n tasks; per task: T, prio (larger = higher, ties by index), gpu_prio (the priority of the
+ * task's GPU segments under the GCAPS policy, Sec. 5.3), core, offset, and the CSR segment
  * arrays restricted to this taskset (cseg_off/gseg_off have n+1 entries, relative to the given
  * cseg/gm/ge arrays).  policy 0 = GCAPS, 1 = RR; busy 0/1; L = RR slice in ticks.
  * Simulates ticks [0, horizon).  max_resp[i] receives the largest response time of a job of
  * task i that COMPLETED inside the horizon (0 if none), unfinished[i] the age of a job still
  * running at the horizon (0 if none).  Returns 0, or -1 if the taskset does not fit the limits.
  */
-int des_simulate(int n, const int64_t *T, const int64_t *prio, const int64_t *core,
-                 const int64_t *offset, const int64_t *cseg_off, const int64_t *cseg,
-                 const int64_t *gseg_off, const int64_t *gm, const int64_t *ge, int policy,
-                 int busy, int64_t L, int64_t horizon, int64_t *max_resp, int64_t *unfinished) {
+int des_simulate_gp(int n, const int64_t *T, const int64_t *prio, const int64_t *gpu_prio,
+                    const int64_t *core, const int64_t *offset, const int64_t *cseg_off,
+                    const int64_t *cseg, const int64_t *gseg_off, const int64_t *gm,
+                    const int64_t *ge, int policy, int busy, int64_t L, int64_t horizon,
+                    int64_t *max_resp, int64_t *unfinished) {
   if (n < 1 || n > SIM_MAX_TASKS) return -1;
   job_shape_t shape[SIM_MAX_TASKS];
   for (int i = 0; i < n; ++i) {
@@ -109,7 +111,7 @@ int des_simulate(int n, const int64_t *T, const int64_t *prio, const int64_t *co
     if (policy == 0) {
       for (int i = 0; i < n; ++i) {
         if (!active[i] || shape[i].kind[phase[i]] != 1) continue;
-        if (gpu_owner < 0 || prio[i] > prio[gpu_owner]) gpu_owner = i;
+        if (gpu_owner < 0 || gpu_prio[i] > gpu_prio[gpu_owner]) gpu_owner = i;
       }
     } else {
       int cur_ready = rr_cur >= 0 && active[rr_cur] && shape[rr_cur].kind[phase[rr_cur]] == 1;
@@ -158,4 +160,13 @@ int des_simulate(int n, const int64_t *T, const int64_t *prio, const int64_t *co
     else if (backlog[i] > 0) unfinished[i] = horizon - (next_rel[i] - T[i] * backlog[i]);
   }
   return 0;
+}
+
+/* The same with the GPU arbitrated by the tasks' CPU priorities. */
+int des_simulate(int n, const int64_t *T, const int64_t *prio, const int64_t *core,
+                 const int64_t *offset, const int64_t *cseg_off, const int64_t *cseg,
+                 const int64_t *gseg_off, const int64_t *gm, const int64_t *ge, int policy,
+                 int busy, int64_t L, int64_t horizon, int64_t *max_resp, int64_t *unfinished) {
+  return des_simulate_gp(n, T, prio, prio, core, offset, cseg_off, cseg, gseg_off, gm, ge, policy,
+                         busy, L, horizon, max_resp, unfinished);
 }

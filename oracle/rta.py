@@ -17,6 +17,7 @@ POLICY_GCAPS = 0
 POLICY_RR = 1
 FLAG_BUSY = 0x100
 FLAG_LITERAL = 0x200
+FLAG_ASSIGN = 0x400
 
 SCHED_NO, SCHED_YES, SCHED_INVALID = 0, 1, 2
 WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID = -1, -2, -3, -4
@@ -109,3 +110,46 @@ def validate(batch) -> np.ndarray:
     lib.oracle_validate_range(ctypes.byref(s), 0, n_tasksets,
                               err.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)))
     return err
+
+
+_gp_lib = None
+
+
+def _load_gpu_prio():
+    global _gp_lib
+    if _gp_lib is None:
+        lib = ctypes.CDLL(_build.build("gpu_prio_oracle"))
+        lib.oracle_gpu_prio_range.argtypes = [
+            ctypes.POINTER(_Tasksets), ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int64,
+            ctypes.c_int64, _p64, _p64, _p64, ctypes.POINTER(ctypes.c_uint8)]
+        lib.oracle_gpu_prio_range.restype = ctypes.c_int
+        _gp_lib = lib
+    return _gp_lib
+
+
+def analyse_gpu_priority(batch, flags: int = 0, overhead_us: int = 0, gpu_priority=None,
+                         iter_cap: int = ITER_CAP):
+    """GCAPS analysis with separate GPU-segment priorities (paper Sec. 5.3 / 6.4).
+
+    ``flags``: ``FLAG_BUSY``, ``FLAG_LITERAL``, ``FLAG_ASSIGN``.  With ``FLAG_ASSIGN`` the GPU
+    priorities are searched (Audsley) and ``gpu_priority`` is ignored; otherwise ``gpu_priority``
+    (int64 per task, larger = higher) is analysed as given.  Returns
+    ``(wcrt, sched, gpu_priority_out)``.
+    """
+    lib = _load_gpu_prio()
+    s, keep = _pack(batch)
+    n_tasksets = keep[0].shape[0] - 1
+    wcrt = np.full(s.n_tasks, WCRT_INVALID, np.int64)
+    sched = np.full(n_tasksets, SCHED_INVALID, np.uint8)
+    out_gp = np.zeros(s.n_tasks, np.int64)
+    gp_in = None
+    if gpu_priority is not None:
+        gp_in = np.ascontiguousarray(gpu_priority, dtype=np.int64)
+        assert gp_in.shape[0] == s.n_tasks
+    rc = lib.oracle_gpu_prio_range(
+        ctypes.byref(s), 0, n_tasksets, flags, overhead_us, iter_cap,
+        gp_in.ctypes.data_as(_p64) if gp_in is not None else None, out_gp.ctypes.data_as(_p64),
+        wcrt.ctypes.data_as(_p64), sched.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)))
+    if rc != 0:
+        raise ValueError("oracle: arguments outside the input domain")
+    return wcrt, sched, out_gp

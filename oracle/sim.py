@@ -16,25 +16,28 @@ def _load():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(_build.build("des_sim"))
-        lib.des_simulate.argtypes = [ctypes.c_int] + [_p64] * 9 + [
+        lib.des_simulate_gp.argtypes = [ctypes.c_int] + [_p64] * 10 + [
             ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_int64, _p64, _p64]
-        lib.des_simulate.restype = ctypes.c_int
+        lib.des_simulate_gp.restype = ctypes.c_int
         _lib = lib
     return _lib
 
 
 def simulate(batch, t: int, offsets: Sequence[int], policy: int, busy: bool, timeslice: int,
-             horizon: int) -> Tuple[np.ndarray, np.ndarray]:
+             horizon: int, gpu_priority=None) -> Tuple[np.ndarray, np.ndarray]:
     """Simulates taskset ``t`` of ``batch`` for ``horizon`` ticks.
 
     Returns ``(max_resp, unfinished)`` per task: the largest response time of a completed job and
-    the age of a job still in progress at the horizon (0 if none).
+    the age of a job still in progress at the horizon (0 if none).  ``gpu_priority`` (per task of
+    the taskset) arbitrates the GPU under GCAPS instead of the CPU priorities.
     """
     lib = _load()
     a, b = int(batch.task_off[t]), int(batch.task_off[t + 1])
     n = b - a
     c = lambda x: np.ascontiguousarray(x, dtype=np.int64)
     T, prio, core = c(batch.period[a:b]), c(batch.priority[a:b]), c(batch.core[a:b])
+    gprio = prio if gpu_priority is None else c(gpu_priority)  # GPU-segment priorities (GCAPS)
+    assert gprio.shape[0] == n
     off = c(offsets)
     assert off.shape[0] == n
     c_off = c(batch.cseg_off[a:b + 1] - batch.cseg_off[a])
@@ -45,7 +48,7 @@ def simulate(batch, t: int, offsets: Sequence[int], policy: int, busy: bool, tim
     max_resp = np.zeros(n, np.int64)
     unfinished = np.zeros(n, np.int64)
     p = lambda x: x.ctypes.data_as(_p64)
-    rc = lib.des_simulate(n, p(T), p(prio), p(core), p(off), p(c_off), p(cs), p(g_off), p(gm),
+    rc = lib.des_simulate_gp(n, p(T), p(prio), p(gprio), p(core), p(off), p(c_off), p(cs), p(g_off), p(gm),
                           p(ge), policy, 1 if busy else 0, timeslice, horizon, p(max_resp),
                           p(unfinished))
     if rc != 0:
