@@ -49,6 +49,7 @@ extern "C" {
 #define GCAPS_POLICY_RR 1
 #define GCAPS_RTA_BUSY 0x100
 #define GCAPS_RTA_LITERAL 0x200
+#define GCAPS_RTA_ASSIGN 0x400 /* only for gcaps_rta_gpu_priority_batch: search the GPU priorities */
 
 /* ---- values written to out_sched[t] --------------------------------------------------------- */
 #define GCAPS_SCHED_NO 0      /* some task's bound exceeds its deadline (or hit ITER_LIMIT)      */
@@ -155,6 +156,38 @@ size_t gcaps_rta_workspace_bytes(int64_t n_tasksets);
 int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
                          int64_t timeslice_us, int64_t ctx_switch_overhead_us, int64_t *out_wcrt,
                          uint8_t *out_sched);
+
+/*
+ * gcaps_rta_gpu_priority_batch -- the GCAPS analysis with a separate priority for the GPU
+ * segments of every task (Sec. 5.3 "Separate Priority for GPU Segments", Sec. 6.4 "Analysis for
+ * GPU Priority Assignment").  hp(tau_i) of Lemmas 10, 11 and 13 becomes the set of tasks with a
+ * higher GPU-segment priority, hpp(tau_i) keeps its meaning (same core, higher CPU priority),
+ * and every jitter uses D_h in place of R_h, so each task is analysed on its own.
+ *
+ *   flags               GCAPS_RTA_BUSY, GCAPS_RTA_LITERAL (as for gcaps_rta_batch), GCAPS_RTA_ASSIGN
+ *   runlist_update_us   epsilon (Def. 2), 0..MAX_TIME
+ *   gpu_priority        DEVICE, [ts->n_tasks], larger = higher, ties by position; used unless
+ *                       GCAPS_RTA_ASSIGN is set (may be NULL then).  Within one core the order
+ *                       of the GPU priorities must equal the order of the CPU priorities (the
+ *                       paper's deadlock rule); a taskset that breaks it is GCAPS_SCHED_INVALID.
+ *   out_gpu_priority    DEVICE, [ts->n_tasks]; required with GCAPS_RTA_ASSIGN, else optional (a
+ *                       copy of gpu_priority).  With GCAPS_RTA_ASSIGN it receives the levels the
+ *                       Audsley-style search of Sec. 5.3 found: 1 (lowest) .. n (highest), 0 for
+ *                       tasks it could not place.  Levels are filled from the lowest; at each
+ *                       level the unplaced tasks are tried from the lowest CPU priority upwards
+ *                       (only a task with no unplaced task of lower CPU priority on its core is a
+ *                       candidate) and the first one whose bound meets its deadline with all
+ *                       other unplaced tasks above it takes the level.
+ *   out_wcrt            DEVICE, [ts->n_tasks]: the task's bound, GCAPS_WCRT_MISS (also: never
+ *                       placed) or GCAPS_WCRT_ITER_LIMIT; nothing is SKIPPED here
+ *   out_sched           DEVICE, [n_tasksets]: 1 if every task has a bound within its deadline
+ *
+ * Asynchronous on `stream`, no workspace, no allocation.  Same return codes as gcaps_rta_batch.
+ */
+int gcaps_rta_gpu_priority_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int flags,
+                                 int64_t runlist_update_us, const int64_t *gpu_priority,
+                                 int64_t *out_gpu_priority, int64_t *out_wcrt, uint8_t *out_sched,
+                                 void *stream);
 
 /*
  * gcaps_rta_batch_host_multi -- gcaps_rta_batch_host for several analyses of the same batch (the

@@ -19,6 +19,7 @@ POLICY_GCAPS = 0
 POLICY_RR = 1
 BUSY = 0x100
 LITERAL = 0x200
+ASSIGN = 0x400
 
 SCHED_NO, SCHED_YES, SCHED_INVALID = 0, 1, 2
 WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID = -1, -2, -3, -4
@@ -31,7 +32,7 @@ STATIC_MAX_TASKSETS = 65536
 EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host",
            "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
            "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static",
-           "gcaps_rta_batch_host_multi")
+           "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch")
 
 _p64 = ctypes.POINTER(ctypes.c_int64)
 
@@ -80,6 +81,10 @@ def load_library(path: Optional[str] = None):
             ctypes.c_int64, ctypes.c_int64, ctypes.POINTER(ctypes.c_void_p),
             ctypes.POINTER(ctypes.c_void_p)]
         lib.gcaps_rta_batch_host_multi.restype = ctypes.c_int
+        lib.gcaps_rta_gpu_priority_batch.argtypes = [
+            ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_void_p,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.gcaps_rta_gpu_priority_batch.restype = ctypes.c_int
         lib.gcaps_rta_release_host.argtypes = []
         lib.gcaps_rta_release_host.restype = None
         lib.gcaps_rta_validate.argtypes = [ctypes.POINTER(CTasksets), ctypes.c_int64,
@@ -174,6 +179,27 @@ def rta_batch_static(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, 
                                         st.cuda_stream)
     _check(rc)
     return out_wcrt, out_sched
+
+
+def rta_gpu_priority(ts: DeviceTasksets, flags: int = 0, overhead_us: int = 0, gpu_priority=None,
+                     stream=None):
+    """gcaps_rta_gpu_priority_batch: GCAPS with separate GPU-segment priorities.  ``gpu_priority``
+    is an int64 CUDA tensor per task, or None together with ``ASSIGN`` in ``flags`` to search the
+    priorities.  Returns ``(out_wcrt, out_sched, out_gpu_priority)`` CUDA tensors."""
+    import torch
+    lib = load_library()
+    dev = ts.t["task_off"].device
+    with torch.cuda.device(dev):
+        out_wcrt = torch.full((ts.n_tasks,), WCRT_INVALID, dtype=torch.int64, device=dev)
+        out_sched = torch.full((max(ts.n_tasksets, 0),), SCHED_INVALID, dtype=torch.uint8, device=dev)
+        out_gp = torch.zeros(ts.n_tasks, dtype=torch.int64, device=dev)
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        rc = lib.gcaps_rta_gpu_priority_batch(
+            ctypes.byref(ts.c), ts.n_tasksets, flags, overhead_us,
+            gpu_priority.data_ptr() if gpu_priority is not None else None, out_gp.data_ptr(),
+            out_wcrt.data_ptr(), out_sched.data_ptr(), st.cuda_stream)
+    _check(rc)
+    return out_wcrt, out_sched, out_gp
 
 
 def rta_validate(ts: DeviceTasksets, stream=None):

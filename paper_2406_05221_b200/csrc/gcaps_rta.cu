@@ -1073,6 +1073,207 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kern
 }
 
 // ---------------------------------------------------------------------------------------------
+// separate GPU-segment priorities (Sec. 5.3, Sec. 6.4): one warp per taskset, exact arithmetic
+// ---------------------------------------------------------------------------------------------
+struct GpSmem {  // by position
+  u64 T[GCAPS_RTA_MAX_TASKS], D[GCAPS_RTA_MAX_TASKS];
+  u64 A[GCAPS_RTA_MAX_TASKS];     // C + G^m
+  u64 Ge[GCAPS_RTA_MAX_TASKS];    // G^e
+  u64 Star[GCAPS_RTA_MAX_TASKS];  // 2 * eps * eta^g
+  i64 key[GCAPS_RTA_MAX_TASKS];   // priorities while ranking
+  int core[GCAPS_RTA_MAX_TASKS];
+  int eta[GCAPS_RTA_MAX_TASKS];
+  short cpu_rank[GCAPS_RTA_MAX_TASKS], gpu_rank[GCAPS_RTA_MAX_TASKS];
+  short by_cpu_rank[GCAPS_RTA_MAX_TASKS];  // CPU rank -> position
+  unsigned char above[GCAPS_RTA_MAX_TASKS];  // 1: has a higher GPU priority than the task analysed
+};
+
+// Bound of task i when the tasks flagged in s.above[] have a higher GPU-segment priority: the
+// recurrence of Sec. 6.3 with hp() by GPU priority and D_h in the jitters (Sec. 6.4).  Lanes over
+// the other tasks.  Returns the bound, GCAPS_WCRT_MISS or GCAPS_WCRT_ITER_LIMIT (warp-uniform).
+__device__ i64 gp_bound(const GpSmem &s, int n, int i, bool busy, bool literal, u64 eps, int lane) {
+  const bool gi = s.eta[i] > 0;
+  const u64 base = s.A[i] + s.Ge[i] + s.Star[i] + ((u64)s.eta[i] + 1) * eps;  // C_i + G*_i + B^C_i
+  const u64 Di = s.D[i];
+  const int core_i = s.core[i], rank_i = s.cpu_rank[i];
+  u64 R = base;
+  i64 sweeps = 0;
+  for (;;) {
+    if (R > Di) return GCAPS_WCRT_MISS;
+    if (sweeps >= GCAPS_RTA_ITER_CAP) return GCAPS_WCRT_ITER_LIMIT;
+    sweeps += 1;
+    u64 part = 0;
+    for (int h = lane; h < n; h += 32) {
+      if (h == i) continue;
+      const bool hpp = s.core[h] == core_i && s.cpu_rank[h] < rank_i;
+      const bool hp_gpu = s.above[h] != 0 && !hpp;
+      const bool gh = s.eta[h] > 0;
+      const u64 Th = s.T[h];
+      const u64 Jc = s.D[h] - s.A[h], Jg = s.D[h] - s.Ge[h];
+      u64 term = 0;
+      if (!busy) {
+        if (hpp && !gh) term = sat_mul(ceil_div64(R, Th), s.A[h]);                  // Lemma 15
+        if (hpp && gh) term = sat_mul(ceil_div64(R + Jc, Th), s.A[h] + s.Star[h]);  // Lemma 15
+        if (hpp && gh && gi) term += sat_mul(ceil_div64(R + Jg, Th), s.Ge[h]);      // Lemma 13
+        if (hp_gpu && gh && gi) term = sat_mul(ceil_div64(R + Jg, Th), s.Ge[h] + s.Star[h]);
+      } else {
+        if (hpp) {
+          u64 W = s.A[h];                                          // Lemma 12
+          if (gh && (gi || !literal)) W += s.Ge[h] + s.Star[h];    // Lemma 10
+          term = sat_mul(ceil_div64(R, Th), W);
+        } else if (hp_gpu && gh) {
+          term = sat_mul(ceil_div64(R + Jg, Th), s.Ge[h] + s.Star[h]);  // Lemmas 10, 11
+        }
+      }
+      part += term;
+    }
+    const u64 next = base + group_sum<32>(part, kFull);
+    if (next == R) return (i64)R;
+    R = next;
+  }
+}
+
+struct GpParams {
+  KParams k;
+  const i64 *gpu_prio_in;
+  i64 *gpu_prio_out;
+  int assign;
+};
+
+__global__ void __launch_bounds__(kBlockThreads) gpu_priority_kernel(GpParams g) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const KParams &p = g.k;
+  const int lane = threadIdx.x & 31;
+  GpSmem &s = reinterpret_cast<GpSmem *>(smem_raw)[threadIdx.x >> 5];
+  const i64 t = (i64)blockIdx.x * (kBlockThreads / 32) + (threadIdx.x >> 5);
+  if (t >= p.n_tasksets) return;
+  const bool busy = (p.policy & GCAPS_RTA_BUSY) != 0, literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
+  const u64 eps = (u64)p.ovh;
+  const i64 a = p.task_off[t], b = p.task_off[t + 1];
+  if (a < 0 || b < a || b > p.n_tasks || b - a > GCAPS_RTA_MAX_TASKS) {
+    if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
+    return;
+  }
+  const int n = (int)(b - a);
+  // ---- stage, validate, aggregate (task model of Sec. 4) ----------------------------------
+  int bad = 0;
+  for (int i = lane; i < n; i += 32) {
+    const i64 k = a + i;
+    const i64 T = p.period[k], D = p.deadline[k], c = p.core[k];
+    if (T < 1 || T > GCAPS_RTA_MAX_TIME) bad |= GCAPS_BAD_PERIOD;
+    if (D < 1 || D > T) bad |= GCAPS_BAD_DEADLINE;
+    if (c < 0 || c > GCAPS_RTA_MAX_CORE) bad |= GCAPS_BAD_CORE;
+    const i64 c0 = p.cseg_off[k], c1 = p.cseg_off[k + 1], g0 = p.gseg_off[k], g1 = p.gseg_off[k + 1];
+    const bool seg_ok = !(c0 < 0 || c1 < c0 || c1 > p.n_csegs || c1 - c0 > GCAPS_RTA_MAX_SEGMENTS ||
+                          g0 < 0 || g1 < g0 || g1 > p.n_gsegs || g1 - g0 > GCAPS_RTA_MAX_SEGMENTS);
+    u64 C = 0, Gm = 0, Ge = 0;
+    if (seg_ok) {
+      for (i64 j = c0; j < c1; ++j) {
+        const i64 w = p.cseg_wcet[j];
+        if (w < 0 || w > GCAPS_RTA_MAX_TIME) bad |= GCAPS_BAD_WCET;
+        C += (u64)w;
+      }
+      for (i64 j = g0; j < g1; ++j) {
+        const i64 m = p.gseg_misc[j], e = p.gseg_exec[j];
+        if (m < 0 || m > GCAPS_RTA_MAX_TIME || e < 0 || e > GCAPS_RTA_MAX_TIME) bad |= GCAPS_BAD_WCET;
+        Gm += (u64)m, Ge += (u64)e;
+      }
+    } else {
+      bad |= GCAPS_BAD_SEG_RANGE;
+    }
+    const int eta = seg_ok ? (int)(g1 - g0) : 0;
+    s.T[i] = (u64)T, s.D[i] = (u64)D, s.A[i] = C + Gm, s.Ge[i] = Ge;
+    s.Star[i] = 2 * eps * (u64)eta;
+    s.core[i] = (int)c, s.eta[i] = eta;
+    s.key[i] = p.priority[k];
+  }
+  bad = group_or<32>(bad, kFull);
+  __syncwarp();
+  if (bad) {
+    for (int i = lane; i < n; i += 32) {
+      p.out_wcrt[a + i] = GCAPS_WCRT_INVALID;
+      if (g.gpu_prio_out) g.gpu_prio_out[a + i] = 0;
+    }
+    if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
+    return;
+  }
+  for (int i = lane; i < n; i += 32) {  // CPU ranks: larger priority first, ties by position
+    const i64 pi = s.key[i];
+    int r = 0;
+    for (int q = 0; q < n; ++q) r += (s.key[q] > pi || (s.key[q] == pi && q < i)) ? 1 : 0;
+    s.cpu_rank[i] = (short)r;
+    s.by_cpu_rank[r] = (short)i;
+  }
+  __syncwarp();
+  int sched = GCAPS_SCHED_YES;
+  if (!g.assign) {
+    for (int i = lane; i < n; i += 32) s.key[i] = g.gpu_prio_in[a + i];
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) {
+      const i64 pi = s.key[i];
+      int r = 0;
+      for (int q = 0; q < n; ++q) r += (s.key[q] > pi || (s.key[q] == pi && q < i)) ? 1 : 0;
+      s.gpu_rank[i] = (short)r;
+    }
+    __syncwarp();
+    int broken = 0;  // same core: the GPU order must equal the CPU order (Sec. 5.3)
+    for (int i = lane; i < n; i += 32)
+      for (int q = 0; q < n; ++q)
+        if (s.core[i] == s.core[q] && s.cpu_rank[q] < s.cpu_rank[i] && s.gpu_rank[q] > s.gpu_rank[i]) broken = 1;
+    if (group_or<32>(broken, kFull)) {
+      for (int i = lane; i < n; i += 32) p.out_wcrt[a + i] = GCAPS_WCRT_INVALID;
+      if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
+      return;
+    }
+    for (int i = 0; i < n; ++i) {
+      for (int q = lane; q < n; q += 32) s.above[q] = s.gpu_rank[q] < s.gpu_rank[i] ? 1 : 0;
+      __syncwarp();
+      const i64 r = gp_bound(s, n, i, busy, literal, eps, lane);
+      if (lane == 0) {
+        p.out_wcrt[a + i] = r;
+        if (g.gpu_prio_out) g.gpu_prio_out[a + i] = g.gpu_prio_in[a + i];
+      }
+      if (r < 0) sched = GCAPS_SCHED_NO;
+      __syncwarp();
+    }
+  } else {
+    // gpu_rank doubles as "unassigned" flag here: -1 while the task has no level yet
+    for (int i = lane; i < n; i += 32) {
+      s.gpu_rank[i] = -1;
+      p.out_wcrt[a + i] = GCAPS_WCRT_MISS;
+      g.gpu_prio_out[a + i] = 0;
+    }
+    __syncwarp();
+    for (int level = 1; level <= n && sched == GCAPS_SCHED_YES; ++level) {
+      bool placed = false;
+      for (int want = n - 1; want >= 0 && !placed; --want) {  // lowest CPU priority first
+        const int c = s.by_cpu_rank[want];
+        if (s.gpu_rank[c] >= 0) continue;
+        int lower = 0;  // an unassigned task of lower CPU priority on the same core bars c
+        for (int q = lane; q < n; q += 32)
+          if (q != c && s.gpu_rank[q] < 0 && s.core[q] == s.core[c] && s.cpu_rank[q] > s.cpu_rank[c]) lower = 1;
+        if (group_or<32>(lower, kFull)) continue;
+        for (int q = lane; q < n; q += 32) s.above[q] = (s.gpu_rank[q] < 0 && q != c) ? 1 : 0;
+        __syncwarp();
+        const i64 r = gp_bound(s, n, c, busy, literal, eps, lane);
+        __syncwarp();
+        if (r >= 0) {
+          placed = true;
+          if (lane == 0) {
+            s.gpu_rank[c] = (short)level;
+            p.out_wcrt[a + c] = r;
+            g.gpu_prio_out[a + c] = (i64)level;
+          }
+          __syncwarp();
+        }
+      }
+      if (!placed) sched = GCAPS_SCHED_NO;
+    }
+  }
+  if (lane == 0) p.out_sched[t] = (uint8_t)sched;
+}
+
+// ---------------------------------------------------------------------------------------------
 // validation kernel: one thread per taskset
 // ---------------------------------------------------------------------------------------------
 __global__ void validate_kernel(KParams p, int32_t *out_err) {
@@ -1349,6 +1550,48 @@ int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int p
   // analysis kernels of this call read.
   return enqueue_batch(p, g_static_scratch_ptr[dev], (size_t)GCAPS_RTA_STATIC_SCRATCH_BYTES,
                        di.sm_count, (cudaStream_t)stream);
+}
+
+int gcaps_rta_gpu_priority_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int flags,
+                                 int64_t runlist_update_us, const int64_t *gpu_priority,
+                                 int64_t *out_gpu_priority, int64_t *out_wcrt, uint8_t *out_sched,
+                                 void *stream) {
+  if (flags & ~(GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL | GCAPS_RTA_ASSIGN)) return GCAPS_ERR_INVALID_ARG;
+  int rc = check_args(ts, n_tasksets, GCAPS_POLICY_GCAPS | (flags & (GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL)),
+                      1, runlist_update_us);
+  if (rc != GCAPS_OK) return rc;
+  const bool assign = (flags & GCAPS_RTA_ASSIGN) != 0;
+  if (n_tasksets == 0) return GCAPS_OK;
+  if (!out_sched || (ts->n_tasks > 0 && (!out_wcrt || (assign ? !out_gpu_priority : !gpu_priority))))
+    return GCAPS_ERR_INVALID_ARG;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != GCAPS_OK) return rc;
+  GpParams g;
+  fill_params(&g.k, ts, n_tasksets, GCAPS_POLICY_GCAPS | (flags & (GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL)), 1,
+              runlist_update_us, out_wcrt, out_sched);
+  g.gpu_prio_in = (const i64 *)gpu_priority;
+  g.gpu_prio_out = (i64 *)out_gpu_priority;
+  g.assign = assign ? 1 : 0;
+  constexpr int kWarps = kBlockThreads / 32;
+  const size_t smem = sizeof(GpSmem) * kWarps;
+  static bool attr_done[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess && !attr_done[dev & 63]) {
+    e = cudaFuncSetAttribute(gpu_priority_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) attr_done[dev & 63] = true;
+  }
+  if (e == cudaSuccess) {
+    const unsigned int grid = (unsigned int)((n_tasksets + kWarps - 1) / kWarps);
+    gpu_priority_kernel<<<grid, kBlockThreads, smem, (cudaStream_t)stream>>>(g);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    return GCAPS_ERR_CUDA;
+  }
+  return GCAPS_OK;
 }
 
 int gcaps_rta_validate(const gcaps_tasksets_t *ts, int64_t n_tasksets, int32_t *out_err,
