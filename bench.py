@@ -178,6 +178,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--ref-sample", type=int, default=100_000)
+    ap.add_argument("--mode", default="policies", choices=["policies", "assign"],
+                    help="policies: GCAPS + RR calls per step (the benchmark); assign: the GCAPS call "
+                         "followed by the GPU-priority search of the paper's Sec. 5.3 on the same batch")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -224,12 +227,19 @@ def main():
     L, ovh = workload.timeslice_us, workload.overhead_us
     stream = torch.cuda.current_stream(dev)
 
+    if args.mode == "assign":
+        policies, names = [binding.POLICY_GCAPS, binding.ASSIGN], ["gcaps", "gpu_priority_search"]
+        args.no_e2e = True
+
     def step(events=None):
         for k, policy in enumerate(policies):
             if events is not None:
                 events[k].record(stream)
-            binding.rta_batch(ts, policy, L, ovh, out_wcrt=out_wcrt, out_sched=out_sched,
-                              workspace=workspace, stream=stream)
+            if args.mode == "assign" and k == 1:
+                binding.rta_gpu_priority(ts, binding.ASSIGN, ovh, None, stream=stream)
+            else:
+                binding.rta_batch(ts, policy, L, ovh, out_wcrt=out_wcrt, out_sched=out_sched,
+                                  workspace=workspace, stream=stream)
         if events is not None:
             events[len(policies)].record(stream)
 
@@ -307,7 +317,7 @@ def main():
                 "best_ms_per_launch": dict(zip(names, best_policy_ms)),
                 "frac_per_policy": {nm: bytes_per_call / (ms * 1e-3) / 1e9 / peak
                                     for nm, ms in zip(names, per_policy_ms)}}
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and args.mode == "policies":
             r = oracle_sample(workload, first, count, args.cpu_budget)
             cpu = {"value": r["tasksets"] / r["seconds"], "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": "first %d tasksets of the workload, both policies, %.1f s, generation excluded"
@@ -338,7 +348,8 @@ def main():
                        "schedulable_fraction_last_policy": sched_frac,
                        "input_checksum": batch.checksum() if count <= 200_000 else None},
             "clocks": clocks, "e2e": e2e,
-            "gpu_launches": args.steps * len(policies) * LAUNCHES_PER_CALL,
+            "gpu_launches": args.steps * (len(policies) * LAUNCHES_PER_CALL if args.mode == "policies"
+                                          else LAUNCHES_PER_CALL + 1),
             "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
         }
         print(json.dumps(line))
