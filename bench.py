@@ -57,7 +57,8 @@ def captured_traffic(workload_name, policy_name, tasksets):
         return None
     if digest != CAPTURED_TRAFFIC["source_sha256"] or workload_name != CAPTURED_TRAFFIC["workload"]:
         return None
-    return CAPTURED_TRAFFIC["bytes_per_taskset"][policy_name] * tasksets
+    per_taskset = CAPTURED_TRAFFIC["bytes_per_taskset"].get(policy_name)
+    return per_taskset * tasksets if per_taskset is not None else None
 
 
 def measured_peaks():
@@ -178,9 +179,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--ref-sample", type=int, default=100_000)
-    ap.add_argument("--mode", default="policies", choices=["policies", "assign"],
+    ap.add_argument("--mode", default="policies", choices=["policies", "assign", "sweep"],
                     help="policies: GCAPS + RR calls per step (the benchmark); assign: the GCAPS call "
-                         "followed by the GPU-priority search of the paper's Sec. 5.3 on the same batch")
+                         "followed by the GPU-priority search of the paper's Sec. 5.3 on the same batch; "
+                         "sweep: all (timeslice, overhead) pairs of the workload, once as one fused "
+                         "gcaps_rta_sweep_batch call and once as one gcaps_rta_batch call per pair")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -230,6 +233,18 @@ def main():
     if args.mode == "assign":
         policies, names = [binding.POLICY_GCAPS, binding.ASSIGN], ["gcaps", "gpu_priority_search"]
         args.no_e2e = True
+    pairs = None
+    if args.mode == "sweep":
+        # two legs per step: [0] the fused call, [1] one call per pair; the policy is the workload's
+        # last one (round robin for the driver-model workload)
+        sweep_policy = policies[-1]
+        tl = getattr(workload, "timeslices", None) or [L]
+        ol = getattr(workload, "overheads", None) or [0, 25, 50, 100, 200]
+        pairs = [(a, b) for a in tl for b in ol]
+        policies, names = ["fused", "separate"], ["fused_sweep", "one_call_per_pair"]
+        sweep_sched = torch.empty((len(pairs), ts.n_tasksets), dtype=torch.uint8, device=dev)
+        sweep_wcrt = torch.empty((len(pairs), ts.n_tasks), dtype=torch.int64, device=dev)
+        args.no_e2e = True
 
     def step(events=None):
         for k, policy in enumerate(policies):
@@ -237,6 +252,14 @@ def main():
                 events[k].record(stream)
             if args.mode == "assign" and k == 1:
                 binding.rta_gpu_priority(ts, binding.ASSIGN, ovh, None, stream=stream)
+            elif args.mode == "sweep" and k == 0:
+                binding.rta_sweep(ts, sweep_policy, [a for a, _ in pairs], [b for _, b in pairs],
+                                  out_wcrt=sweep_wcrt, out_sched=sweep_sched, workspace=workspace,
+                                  stream=stream)
+            elif args.mode == "sweep":
+                for q, (a, b) in enumerate(pairs):
+                    binding.rta_batch(ts, sweep_policy, a, b, out_wcrt=sweep_wcrt[q],
+                                      out_sched=sweep_sched[q], workspace=workspace, stream=stream)
             else:
                 binding.rta_batch(ts, policy, L, ovh, out_wcrt=out_wcrt, out_sched=out_sched,
                                   workspace=workspace, stream=stream)
@@ -269,10 +292,13 @@ def main():
     total_ms = ev[0][0].elapsed_time(ev[-1][-1])
     per_policy_ms = [statistics.mean(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(len(policies))]
     best_policy_ms = [min(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(len(policies))]
-    sched_frac = float((out_sched == 1).float().mean().item()) if count else 0.0
+    flags = sweep_sched[0] if args.mode == "sweep" else out_sched
+    sched_frac = float((flags == 1).float().mean().item()) if count else 0.0
     total_ms = sharding.reduce_scalars([total_ms], "max", dev)[0]
     ms_per_step = total_ms / args.steps
     value = world * count / (ms_per_step * 1e-3)
+    if args.mode == "sweep":  # taskset analyses per second of the fused call alone
+        value = world * count * len(pairs) / (per_policy_ms[0] * 1e-3)
 
     # ---- end to end through the host-buffer entry point (copies inside the timed region) -----
     e2e = None
@@ -301,10 +327,12 @@ def main():
     # ---- the oracle beside it, and the roofline of the dominant launch ------------------------
     cpu = None
     bytes_per_call = batch.input_bytes() + batch.output_bytes()
+    if args.mode == "sweep":  # inputs once, outputs once per pair
+        bytes_per_call = batch.input_bytes() + len(pairs) * batch.output_bytes()
     peak, peak_kind = measured_peaks()
     roof = None
     if rank == 0:
-        dom = int(np.argmax(per_policy_ms))
+        dom = 0 if args.mode == "sweep" else int(np.argmax(per_policy_ms))
         achieved = bytes_per_call / (per_policy_ms[dom] * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak,
@@ -342,13 +370,15 @@ def main():
             "config": {"workload": workload.name, "note": workload.note, "tasksets_per_gpu": count,
                        "tasks": ts.n_tasks, "policies": names, "mode": "self-suspension",
                        "timeslice_us": L, "overhead_us": ovh,
-                       "analyses_per_taskset_per_step": len(policies),
+                       "analyses_per_taskset_per_step": len(pairs) if pairs else len(policies),
+                       "sweep_pairs": pairs,
                        "l2": "inputs (%.2f GB per call) against a 126 MB L2; no flush between steps"
                              % (batch.input_bytes() / 1e9),
                        "schedulable_fraction_last_policy": sched_frac,
                        "input_checksum": batch.checksum() if count <= 200_000 else None},
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": args.steps * (len(policies) * LAUNCHES_PER_CALL if args.mode == "policies"
+                                          else (1 + len(pairs)) * LAUNCHES_PER_CALL if args.mode == "sweep"
                                           else LAUNCHES_PER_CALL + 1),
             "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
         }

@@ -204,6 +204,29 @@ int gcaps_rta_batch_host_multi(const gcaps_tasksets_t *ts, int64_t n_tasksets, c
                                int64_t *const *out_wcrt, uint8_t *const *out_sched);
 
 /*
+ * gcaps_rta_sweep_batch -- one device-resident batch analysed under several (timeslice, overhead)
+ * pairs in a single pass.  The paper's experiments re-run the same generated tasksets while one
+ * parameter of the analysis varies (Sec. 7.1; L of Eq. 3, theta of Def. 1 and epsilon of Def. 2
+ * are such parameters); doing that with gcaps_rta_batch reads every taskset once per pair.  Here
+ * each taskset is read, ordered and aggregated once and then goes through the recurrence of
+ * gcaps_rta_batch once per pair.  Results are those of n_points separate gcaps_rta_batch calls.
+ *
+ *   n_points                1 .. GCAPS_RTA_MAX_SWEEP
+ *   timeslice_us            HOST array [n_points]: L of pair q (RR only; may be NULL for GCAPS)
+ *   ctx_switch_overhead_us  HOST array [n_points]: theta (RR) or epsilon (GCAPS) of pair q
+ *   out_wcrt                DEVICE, [n_points][ts->n_tasks] (pair-major), or NULL when only the
+ *                           schedulable flags are wanted
+ *   out_sched               DEVICE, [n_points][n_tasksets] (pair-major)
+ *   policy, workspace, stream, return codes, asynchrony: as for gcaps_rta_batch; the two host
+ *   arrays are read before the call returns.
+ */
+#define GCAPS_RTA_MAX_SWEEP 32
+int gcaps_rta_sweep_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy, int n_points,
+                          const int64_t *timeslice_us, const int64_t *ctx_switch_overhead_us,
+                          int64_t *out_wcrt, uint8_t *out_sched, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
+/*
  * gcaps_rta_batch_static -- gcaps_rta_batch for callers that are not able to allocate device
  * memory.  (The paper has no counterpart: this is a convenience of this library, not a step of
  * the analysis.)

@@ -100,6 +100,23 @@ def analyse(batch, policy: int, timeslice_us: int = 1024, overhead_us: int = 0,
     return wcrt, sched, counts
 
 
+def analyse_sweep(batch, policy: int, timeslices_us, overheads_us, iter_cap: int = ITER_CAP):
+    """The same batch under several ``(timeslice, overhead)`` pairs -- the paper's experiments
+    re-run one set of tasksets while a parameter varies (Sec. 7.1).  By definition this is one
+    independent ``analyse`` per pair, and that is all this function does.
+
+    Returns ``(wcrt, sched)`` of shapes ``[n_params, n_tasks]`` and ``[n_params, n_tasksets]``.
+    """
+    assert len(timeslices_us) == len(overheads_us)
+    n_tasksets = np.asarray(batch.task_off).shape[0] - 1
+    n_tasks = np.asarray(batch.period).shape[0]
+    wcrt = np.full((len(timeslices_us), n_tasks), WCRT_INVALID, np.int64)
+    sched = np.full((len(timeslices_us), n_tasksets), SCHED_INVALID, np.uint8)
+    for q, (L, ovh) in enumerate(zip(timeslices_us, overheads_us)):
+        analyse(batch, policy, int(L), int(ovh), iter_cap=iter_cap, out=(wcrt[q], sched[q]))
+    return wcrt, sched
+
+
 def validate(batch) -> np.ndarray:
     """Per-taskset domain check; 0 = valid, else a bit mask (1 task range, 2 segment range,
     4 period, 8 deadline, 16 core, 32 WCET)."""

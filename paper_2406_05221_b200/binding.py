@@ -28,11 +28,12 @@ MAX_TIME = 1 << 40
 
 OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NO_DEVICE, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5
 STATIC_MAX_TASKSETS = 65536
+MAX_SWEEP = 32
 
 EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host",
            "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
            "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static",
-           "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch")
+           "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch", "gcaps_rta_sweep_batch")
 
 _p64 = ctypes.POINTER(ctypes.c_int64)
 
@@ -85,6 +86,10 @@ def load_library(path: Optional[str] = None):
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_void_p,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         lib.gcaps_rta_gpu_priority_batch.restype = ctypes.c_int
+        lib.gcaps_rta_sweep_batch.argtypes = [
+            ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int, _p64, _p64,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        lib.gcaps_rta_sweep_batch.restype = ctypes.c_int
         lib.gcaps_rta_release_host.argtypes = []
         lib.gcaps_rta_release_host.restype = None
         lib.gcaps_rta_validate.argtypes = [ctypes.POINTER(CTasksets), ctypes.c_int64,
@@ -152,6 +157,34 @@ def rta_batch(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, overhea
         rc = lib.gcaps_rta_batch(ctypes.byref(ts.c), ts.n_tasksets, policy, timeslice_us, overhead_us,
                                  out_wcrt.data_ptr(), out_sched.data_ptr(), workspace.data_ptr(),
                                  workspace.numel(), st.cuda_stream)
+    _check(rc)
+    return out_wcrt, out_sched
+
+
+def rta_sweep(ts: DeviceTasksets, policy: int, timeslices_us, overheads_us, want_wcrt: bool = True,
+              out_wcrt=None, out_sched=None, workspace=None, stream=None):
+    """gcaps_rta_sweep_batch: the resident batch under every ``(timeslice, overhead)`` pair in one
+    pass.  Returns ``(out_wcrt, out_sched)`` CUDA tensors of shapes ``[n_points, n_tasks]`` (None
+    with ``want_wcrt=False``) and ``[n_points, n_tasksets]``."""
+    import torch
+    lib = load_library()
+    dev = ts.t["task_off"].device
+    k = len(overheads_us)
+    Ls = (ctypes.c_int64 * k)(*[int(x) for x in timeslices_us]) if timeslices_us is not None else None
+    ov = (ctypes.c_int64 * k)(*[int(x) for x in overheads_us])
+    with torch.cuda.device(dev):
+        if out_wcrt is None and want_wcrt:
+            out_wcrt = torch.empty((k, ts.n_tasks), dtype=torch.int64, device=dev)
+        if out_sched is None:
+            out_sched = torch.empty((k, max(ts.n_tasksets, 0)), dtype=torch.uint8, device=dev)
+        need = workspace_bytes(ts.n_tasksets)
+        if workspace is None:
+            workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        rc = lib.gcaps_rta_sweep_batch(ctypes.byref(ts.c), ts.n_tasksets, policy, k, Ls, ov,
+                                       out_wcrt.data_ptr() if out_wcrt is not None else None,
+                                       out_sched.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                       st.cuda_stream)
     _check(rc)
     return out_wcrt, out_sched
 

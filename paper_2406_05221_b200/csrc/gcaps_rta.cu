@@ -70,6 +70,18 @@ struct KParams {
   unsigned int *perm;       // [n_tasksets]
 };
 
+// The (timeslice, overhead) pairs of a fused sweep: one staging and aggregation of a taskset,
+// one analysis per pair.  Passed to the sweep kernels by value.
+struct SweepPoint {
+  i64 L, ovh;
+  u32 l_mode, l_magic, l_shift, pad;  // division by L in the 32-bit path, as in KParams
+};
+struct SweepArgs {
+  int n;        // pairs, 1 .. GCAPS_RTA_MAX_SWEEP
+  i64 max_ovh;  // largest overhead of the sweep
+  SweepPoint q[GCAPS_RTA_MAX_SWEEP];
+};
+
 __device__ __forceinline__ int size_bin(i64 n) {
   if (n <= 8) return 0;  // also negative / broken ranges: rejected by the analysis kernel
   if (n <= 16) return 1;
@@ -271,7 +283,8 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
   const int n_gpu = group_sum_int<LPT>(n_gpu_lane, mask);  // N_g
   __syncwarp(mask);
   if (bad) {
-    for (int i = lane; i < n; i += LPT) p.out_wcrt[a + i] = GCAPS_WCRT_INVALID;
+    if (p.out_wcrt)
+      for (int i = lane; i < n; i += LPT) p.out_wcrt[a + i] = GCAPS_WCRT_INVALID;
     if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
     return;
   }
@@ -360,7 +373,8 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
     }
   }
   __syncwarp(mask);
-  for (int i = lane; i < n; i += LPT) p.out_wcrt[a + i] = s.prio_out[i];
+  if (p.out_wcrt)
+    for (int i = lane; i < n; i += LPT) p.out_wcrt[a + i] = s.prio_out[i];
   if (lane == 0) p.out_sched[t] = (uint8_t)sched;
   __syncwarp(mask);
 }
@@ -558,9 +572,13 @@ __device__ __forceinline__ void prefix_step(const i64 *__restrict__ X0, const i6
 // Then every task's values move through shared memory to the lane that owns its rank, so that the
 // interferers of the task of rank `pos` sit in lanes (pos-1) % LPT downwards of slots up to
 // (pos-1) / LPT and higher slots can be skipped.
-template <int LPT, int SLOTS, int MODE>
+//
+// SWEEP: the taskset is staged, ordered and aggregated once and then analysed under every
+// (timeslice, overhead) pair of `sw`; pair q writes out_wcrt + q * n_tasks (skipped when out_wcrt
+// is null) and out_sched + q * n_tasksets.
+template <int LPT, int SLOTS, int MODE, bool SWEEP = false>
 __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane,
-                                             unsigned int gmask) {
+                                             unsigned int gmask, const SweepArgs *sw = nullptr) {
   typedef FastLayout<LPT, SLOTS> Lay;
   constexpr int kLog = LPT == 32 ? 5 : LPT == 16 ? 4 : 3;  // log2 of the lanes per taskset
   constexpr int MAXN = Lay::MAXN, CAP = Lay::CAP;
@@ -711,9 +729,37 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     bad |= A[s] >> 26;
   }
   __syncwarp(gmask);
-  if (!kGcaps) {  // Eq. 3: slices of every pure GPU part, summed per task (values already checked)
+  // ---- what does not depend on the timeslice or the overhead ---------------------------------
+  int n_gpu = 0;  // N_g
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(gmask, eta[s] > 0));
+  if (kGcaps) {  // 2 * eps * eta must stay below 2^26 (eta < 64, eps < 2^20: no overflow here)
+    const u32 ovh_max = SWEEP ? (u32)sw->max_ovh : (u32)p.ovh;
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) bad |= (2 * ovh_max * eta[s]) >> 26;
+  }
+  if (__any_sync(gmask, bad != 0)) return false;
+  u32 magic[SLOTS], shift[SLOTS];  // reciprocal of T_h by rank, made when the slot is first needed
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) magic[s] = 0, shift[s] = 0;
+  int slots_made = 0;
+  u32 sl[SLOTS];  // RR: slices of the task's pure GPU parts (Eq. 3), by position
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) sl[s] = 0;
+  u32 *Ps = SWEEP ? Q1 : Q0;  // running sums of the slice counts (a sweep keeps Q0 for the exchange)
+  const int n_points = SWEEP ? sw->n : 1;
+  for (int q = 0; q < n_points; ++q) {
+  const i64 L64 = SWEEP ? sw->q[q].L : p.L;
+  const u32 ovh = SWEEP ? (u32)sw->q[q].ovh : (u32)p.ovh;  // the fast path needs eps, theta < 2^20
+  const u32 l_mode = SWEEP ? sw->q[q].l_mode : p.l_mode, l_magic = SWEEP ? sw->q[q].l_magic : p.l_magic;
+  const u32 l_shift = SWEEP ? sw->q[q].l_shift : p.l_shift;
+  i64 *const out_wcrt = SWEEP ? (p.out_wcrt ? p.out_wcrt + (i64)q * p.n_tasks : nullptr) : p.out_wcrt;
+  uint8_t *const out_sched = SWEEP ? p.out_sched + (i64)q * p.n_tasksets : p.out_sched;
+  if (!kGcaps && (!SWEEP || q == 0 || sw->q[q].L != sw->q[q - 1].L)) {
+    // Eq. 3: slices of every pure GPU part, summed per task (values already checked)
     const bool inside = slice_is_inside(gfirst, Ng, pare, p.n_gsegs);
     u32 carry = 0;
+    if (lane == 0) Ps[-1] = 0;
     for (int e0 = 0; e0 < Ng + 1; e0 += Lay::kStep * BG) {
       Quad qe[BG];
       u32 x[BG][4], incl[BG];
@@ -728,11 +774,11 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
         for (int j = 0; j < 4; ++j) {
           // a neighbour's element may be large: keep it below 2^26 so the division stays exact
           const u32 w = (u32)qe[b].v[j] & (kFastLimit - 1);
-          u32 sl;
-          if (p.l_mode == 0) sl = __umulhi(w + (u32)p.L - 1u, p.l_magic) >> p.l_shift;
-          else if (p.l_mode == 1) sl = w;
-          else sl = w > 0 ? 1u : 0u;
-          x[b][j] = sl + (j > 0 ? x[b][j - 1] : 0u);
+          u32 sq;
+          if (l_mode == 0) sq = __umulhi(w + (u32)L64 - 1u, l_magic) >> l_shift;
+          else if (l_mode == 1) sq = w;
+          else sq = w > 0 ? 1u : 0u;
+          x[b][j] = sq + (j > 0 ? x[b][j - 1] : 0u);
         }
         incl[b] = x[b][3];
       }
@@ -748,29 +794,27 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       for (int b = 0; b < BG; ++b) {
         if (e0 + 4 * LPT * b < Ng + 1) {
           const u32 before = incl[b] - x[b][3] + carry;
-          *reinterpret_cast<uint4 *>(Q0 + e0 + 4 * LPT * b + 4 * lane) =
+          *reinterpret_cast<uint4 *>(Ps + e0 + 4 * LPT * b + 4 * lane) =
               make_uint4(x[b][0] + before, x[b][1] + before, x[b][2] + before, x[b][3] + before);
           carry += __shfl_sync(gmask, incl[b], LPT - 1, LPT);
         }
       }
     }
     __syncwarp(gmask);
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) sl[s] = Ps[g1[s] - 1 + pare] - Ps[g0[s] - 1 + pare];
+    __syncwarp(gmask);
   }
   // ---- constants of Eq. 1 that do not depend on R ------------------------------------------
-  int n_gpu = 0;  // N_g
-#pragma unroll
-  for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(gmask, eta[s] > 0));
-  const u32 ovh = (u32)p.ovh;  // the fast path is only entered with eps, theta < 2^20
   u32 base[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     if (kGcaps) {
       S[s] = 2 * ovh * eta[s];                                 // eta < 64: below 2^27
       base[s] = A[s] + Ge[s] + S[s] + (eta[s] + 1) * ovh;        // C_i + G*_i + B^C_i, below 2^29
-      bad |= S[s] >> 26;
     } else {
-      const u64 slices = Q0[g1[s] - 1 + pare] - Q0[g0[s] - 1 + pare];
-      const u64 lt = (u64)p.L + ovh;  // <= 2^41
+      const u64 slices = sl[s];
+      const u64 lt = (u64)L64 + ovh;  // <= 2^41
       u64 B = slices == 0 ? 0 : (lt >= kFastClamp ? kFastClamp : lt * slices);  // < 2^26 * 2^32
       if (B > kFastClamp) B = kFastClamp;
       S[s] = (u32)B;
@@ -779,10 +823,9 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     }
     base[s] = base[s] > 2 * kFastClamp ? 2 * kFastClamp : base[s];
   }
-  if (__any_sync(gmask, bad != 0)) return false;
   __syncwarp(gmask);
   // ---- move every task to the lane that owns its rank -------------------------------------
-  uint4 *xch = reinterpret_cast<uint4 *>(Q0);  // by rank: T, C+G^m, G^e, S  (Q0, Q1 are dead now)
+  uint4 *xch = reinterpret_cast<uint4 *>(Q0);  // by rank: T, C+G^m, G^e, S  (Q0 is dead by now)
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     if (lane + LPT * s < n) {
@@ -792,32 +835,33 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     }
   }
   __syncwarp(gmask);
-  u32 Tm1[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS], core[SLOTS];
+  // by rank from here on: period - 1, C+G^m, G^e, S, the two weights of the analysis' pairs
+  u32 Tm1[SLOTS], Ar[SLOTS], Ger[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS], core[SLOTS];
   bool gpu[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + LPT * s;
     const uint4 x = r < n ? xch[r] : make_uint4(2u, 0u, 0u, 0u);
     const uint4 f = r < n ? info[r] : make_uint4(0u, 0xffffffffu, 0u, 0u);
-    Tm1[s] = x.x - 1, A[s] = x.y, Ge[s] = x.z, S[s] = x.w;
+    const u32 Sr = x.w;
+    Tm1[s] = x.x - 1, Ar[s] = x.y, Ger[s] = x.z;
     core[s] = f.y, pos_of[s] = f.w & 0xffffu, gpu[s] = (f.w & 0x10000u) != 0;
     if (MODE == 0) {
-      Wa[s] = A[s] + (gpu[s] ? S[s] : 0u);  // Lemma 15: C_h, or C_h + G^{m*}_h
-      Wb[s] = gpu[s] ? Ge[s] + S[s] : 0u;   // Lemma 13, other cores: G^{e*}_h
+      Wa[s] = Ar[s] + (gpu[s] ? Sr : 0u);    // Lemma 15: C_h, or C_h + G^{m*}_h
+      Wb[s] = gpu[s] ? Ger[s] + Sr : 0u;     // Lemma 13, other cores: G^{e*}_h
     } else if (MODE == 1) {
-      Wa[s] = A[s];                         // Lemma 12
-      Wb[s] = gpu[s] ? Ge[s] + S[s] : 0u;   // Lemmas 10, 11: G^{e*}_h
+      Wa[s] = Ar[s];                         // Lemma 12
+      Wb[s] = gpu[s] ? Ger[s] + Sr : 0u;     // Lemmas 10, 11: G^{e*}_h
     } else {
-      Wa[s] = A[s];                         // Lemmas 5, 7
-      Wb[s] = gpu[s] ? S[s] : 0u;           // Lemma 4: (L+theta) * slices
+      Wa[s] = Ar[s];                         // Lemmas 5, 7
+      Wb[s] = gpu[s] ? Sr : 0u;              // Lemma 4: (L+theta) * slices
     }
   }
 
   // ---- iterate in rank order ------------------------------------------------------------------
-  u32 magic[SLOTS], shift[SLOTS];         // reciprocal of T_h, made when the slot is first needed
   u32 Jc[SLOTS], Jg[SLOTS];               // jitters with T_h - 1 folded in (ceiling)
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Tm1[s], magic[s] = 0, shift[s] = 0;
+  for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Tm1[s];
   int n_done = n;
   int verdict = 0;
   for (int pos = 0; pos < n; ++pos) {
@@ -825,10 +869,11 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     const u32 Di = f.x, core_i = f.y, base_i = f.z;
     const bool gi = (f.w & 0x10000u) != 0;
     const int smax = (pos - 1) >> kLog;  // -1 for the first task: nothing interferes
-    if ((pos & (LPT - 1)) == 1) {            // the first task that looks at slot smax
+    if (smax >= slots_made) {              // the first task that looks at slot smax
 #pragma unroll
       for (int s = 0; s < SLOTS; ++s)
         if (s == smax) make_reciprocal(Tm1[s] + 1, magic[s], shift[s]);
+      slots_made = smax + 1;
     }
     u32 nu = 0;
     if (MODE == 3) {  // Lemma 4: N_g - |{h in hpp(i): GPU-using}| + 1
@@ -850,7 +895,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
         if (MODE == 0) {
           w1 = same ? Wa[s] : (gi ? Wb[s] : 0u);           // Lemma 15 / Lemma 13 (other cores)
           j1 = same ? Jc[s] : Jg[s];
-          w2 = (same && gi && gpu[s]) ? Ge[s] : 0u;        // Lemma 13 (same core), jitter J^g
+          w2 = (same && gi && gpu[s]) ? Ger[s] : 0u;       // Lemma 13 (same core), jitter J^g
         } else if (MODE == 1) {
           w1 = same ? Wa[s] + ((gi || !literal) ? Wb[s] : 0u) : Wb[s];  // Lemmas 12+10 / 10, 11
           j1 = same ? Tm1[s] : Jg[s];
@@ -904,21 +949,24 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
       if (lane + LPT * s == pos) {
-        p.out_wcrt[a + pos_of[s]] = (i64)R;
-        if (MODE == 0 ? gpu[s] : (MODE == 2 ? (gpu[s] || literal) : false)) Jc[s] = R - A[s] + Tm1[s];
-        Jg[s] = R - Ge[s] + Tm1[s];
+        if (!SWEEP || out_wcrt) out_wcrt[a + pos_of[s]] = (i64)R;
+        if (MODE == 0 ? gpu[s] : (MODE == 2 ? (gpu[s] || literal) : false)) Jc[s] = R - Ar[s] + Tm1[s];
+        Jg[s] = R - Ger[s] + Tm1[s];
       }
     }
   }
   // ---- write the sentinels of the tasks that did not converge ---------------------------------
+  if (!SWEEP || out_wcrt) {
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) {
-    const int r = lane + LPT * s;
-    if (r < n && r >= n_done)
-      p.out_wcrt[a + pos_of[s]] = r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED;
+    for (int s = 0; s < SLOTS; ++s) {
+      const int r = lane + LPT * s;
+      if (r < n && r >= n_done)
+        out_wcrt[a + pos_of[s]] = r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED;
+    }
   }
-  if (lane == 0) p.out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
+  if (lane == 0) out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
   __syncwarp(gmask);
+  }  // next (timeslice, overhead) pair
   return true;
 }
 
@@ -948,8 +996,9 @@ __host__ __device__ constexpr int min_blocks(int slots) {
 // LPT lanes; every group analyses one taskset at a time.  Warps pull chunks of taskset indices
 // from the bin's counter; the index, task range and first segment offsets of the next chunk are
 // fetched while the current one is analysed.
-template <int LPT, int SLOTS, int MODE>
-__device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf, Ahead *ahead) {
+template <int LPT, int SLOTS, int MODE, bool SWEEP = false>
+__device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf, Ahead *ahead,
+                                        const SweepArgs *sw = nullptr) {
   typedef FastLayout<LPT, SLOTS> Lay;
   constexpr int MAXN = LPT * SLOTS;
   constexpr int G = 32 / LPT;  // groups per warp
@@ -959,7 +1008,8 @@ __device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf
   u32 *buf = warp_buf + group * Lay::kWords;
   const unsigned int start = p.hdr->bin_start[bin], count = p.hdr->bin_count[bin];
   if (count == 0) return;
-  const bool fast_call = p.ovh < (1 << 20);  // keeps 2*eps*eta and (eta+1)*eps in 32 bits
+  // keeps 2*eps*eta and (eta+1)*eps in 32 bits
+  const bool fast_call = (SWEEP ? sw->max_ovh : p.ovh) < (1 << 20);
   // tasksets per pull: up to 8 per group when the bin is large, fewer when that would leave warps
   // without work
   const unsigned int n_groups = gridDim.x * (kBlockThreads / 32) * G;
@@ -1024,11 +1074,21 @@ __device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf
           prefetch_l2(p.gseg_misc + me.g_lo + e), prefetch_l2(p.gseg_exec + me.g_lo + e);
         bool done = false;
         if (fast_call && (me.packed >> 31) != 0)
-          done = analyse_fast<LPT, SLOTS, MODE>(p, t, me.a, n, buf, lane, gmask);
+          done = analyse_fast<LPT, SLOTS, MODE, SWEEP>(p, t, me.a, n, buf, lane, gmask, sw);
         __syncwarp(gmask);
-        if (!done) {
+        if (!done && !SWEEP) {
           // the exact path reads task_off again and validates everything itself
           analyse_taskset<LPT, MAXN>(p, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, gmask);
+        }
+        if (!done && SWEEP) {  // the exact path once per (timeslice, overhead) pair
+          for (int q = 0; q < sw->n; ++q) {
+            KParams pq = p;
+            pq.L = sw->q[q].L, pq.ovh = sw->q[q].ovh;
+            pq.out_wcrt = p.out_wcrt ? p.out_wcrt + (i64)q * p.n_tasks : nullptr;
+            pq.out_sched = p.out_sched + (i64)q * p.n_tasksets;
+            analyse_taskset<LPT, MAXN>(pq, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, gmask);
+            __syncwarp(gmask);
+          }
         }
       }
       __syncwarp();
@@ -1070,6 +1130,30 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kern
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
   run_bin<32, SLOTS, MODE>(p, bin, warp_buf, ahead);
+}
+
+// The same launches for a fused sweep: every taskset is read once and analysed under all the
+// (timeslice, overhead) pairs of `sw`.
+template <int MODE>
+__global__ void __launch_bounds__(kBlockThreads, 4)
+rta_small_sweep_kernel(KParams p, const __grid_constant__ SweepArgs sw) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
+  Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
+  run_bin<16, 2, MODE, true>(p, 3, warp_buf, ahead, &sw);
+  run_bin<8, 3, MODE, true>(p, 2, warp_buf, ahead, &sw);
+  run_bin<8, 2, MODE, true>(p, 1, warp_buf, ahead, &sw);
+  run_bin<8, 1, MODE, true>(p, 0, warp_buf, ahead, &sw);
+}
+
+template <int SLOTS, int MODE>
+__global__ void __launch_bounds__(kBlockThreads, (SLOTS <= 4 ? 4 : min_blocks(SLOTS)))
+rta_big_sweep_kernel(KParams p, int bin, const __grid_constant__ SweepArgs sw) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
+  u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
+  Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
+  run_bin<32, SLOTS, MODE, true>(p, bin, warp_buf, ahead, &sw);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1444,7 +1528,33 @@ cudaError_t launch_all_bins(const KParams &p, int sm_count, cudaStream_t st) {
   return e;
 }
 
-int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_count, cudaStream_t st) {
+template <int SLOTS, int MODE>
+cudaError_t launch_big_sweep(const KParams &p, const SweepArgs &sw, int bin, int sm_count, cudaStream_t st) {
+  constexpr int kWarps = kBlockThreads / 32;
+  static int blocks_per_sm[64] = {0};
+  const size_t smem = sizeof(u32) * (bin_warp_words<32, SLOTS>() + kAheadWords) * kWarps;
+  return launch_persistent(rta_big_sweep_kernel<SLOTS, MODE>, blocks_per_sm, smem,
+                           (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p, bin, sw);
+}
+
+template <int MODE>
+cudaError_t launch_all_bins_sweep(const KParams &p, const SweepArgs &sw, int sm_count, cudaStream_t st) {
+  constexpr int kWarps = kBlockThreads / 32;
+  static int blocks_per_sm[64] = {0};
+  const size_t smem = sizeof(u32) * kSmallWarpWords * kWarps;
+  cudaError_t e = launch_persistent(rta_small_sweep_kernel<MODE>, blocks_per_sm, smem,
+                                    (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p, sw);
+  if (e == cudaSuccess) e = launch_big_sweep<2, MODE>(p, sw, 4, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<3, MODE>(p, sw, 5, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<4, MODE>(p, sw, 6, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<6, MODE>(p, sw, 7, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<8, MODE>(p, sw, 8, sm_count, st);
+  return e;
+}
+
+// Plan + analysis launches of one call; `sw` non-null: the fused sweep.
+int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_count, cudaStream_t st,
+                  const SweepArgs *sw = nullptr) {
   if (p.n_tasksets == 0) return GCAPS_OK;
   const size_t need = gcaps_rta_workspace_bytes(p.n_tasksets);
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255u))
@@ -1460,7 +1570,12 @@ int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_cou
   cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) {
     const bool rr = (p.policy & 0xff) == GCAPS_POLICY_RR, busy = (p.policy & GCAPS_RTA_BUSY) != 0;
-    if (!rr && !busy) e = launch_all_bins<0>(p, sm_count, st);
+    if (sw) {
+      if (!rr && !busy) e = launch_all_bins_sweep<0>(p, *sw, sm_count, st);
+      else if (!rr) e = launch_all_bins_sweep<1>(p, *sw, sm_count, st);
+      else if (!busy) e = launch_all_bins_sweep<2>(p, *sw, sm_count, st);
+      else e = launch_all_bins_sweep<3>(p, *sw, sm_count, st);
+    } else if (!rr && !busy) e = launch_all_bins<0>(p, sm_count, st);
     else if (!rr) e = launch_all_bins<1>(p, sm_count, st);
     else if (!busy) e = launch_all_bins<2>(p, sm_count, st);
     else e = launch_all_bins<3>(p, sm_count, st);
@@ -1512,6 +1627,37 @@ int gcaps_rta_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
   KParams p;
   fill_params(&p, ts, n_tasksets, policy, timeslice_us, ctx_switch_overhead_us, out_wcrt, out_sched);
   return enqueue_batch(p, workspace, workspace_bytes, di.sm_count, (cudaStream_t)stream);
+}
+
+int gcaps_rta_sweep_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy, int n_points,
+                          const int64_t *timeslice_us, const int64_t *ctx_switch_overhead_us,
+                          int64_t *out_wcrt, uint8_t *out_sched, void *workspace,
+                          size_t workspace_bytes, void *stream) {
+  if (n_points < 1 || n_points > GCAPS_RTA_MAX_SWEEP || !ctx_switch_overhead_us)
+    return GCAPS_ERR_INVALID_ARG;
+  const bool rr = (policy & 0xff) == GCAPS_POLICY_RR;
+  if (rr && !timeslice_us) return GCAPS_ERR_INVALID_ARG;
+  SweepArgs sw;
+  memset(&sw, 0, sizeof(sw));
+  sw.n = n_points;
+  for (int q = 0; q < n_points; ++q) {
+    const int64_t L = rr ? timeslice_us[q] : 1;
+    int rc = check_args(ts, n_tasksets, policy, L, ctx_switch_overhead_us[q]);
+    if (rc != GCAPS_OK) return rc;
+    KParams one;  // (fills the reciprocal of L exactly as a single call would)
+    fill_params(&one, ts, n_tasksets, policy, L, ctx_switch_overhead_us[q], nullptr, nullptr);
+    sw.q[q].L = one.L, sw.q[q].ovh = one.ovh;
+    sw.q[q].l_mode = one.l_mode, sw.q[q].l_magic = one.l_magic, sw.q[q].l_shift = one.l_shift;
+    if (one.ovh > sw.max_ovh) sw.max_ovh = one.ovh;
+  }
+  if (n_tasksets == 0) return GCAPS_OK;
+  if (!out_sched) return GCAPS_ERR_INVALID_ARG;
+  DeviceInfo di;
+  int rc = device_info(&di);
+  if (rc != GCAPS_OK) return rc;
+  KParams p;
+  fill_params(&p, ts, n_tasksets, policy, sw.q[0].L, sw.q[0].ovh, out_wcrt, out_sched);
+  return enqueue_batch(p, workspace, workspace_bytes, di.sm_count, (cudaStream_t)stream, &sw);
 }
 
 int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
