@@ -18,9 +18,10 @@ POLICY_RR = 1
 FLAG_BUSY = 0x100
 FLAG_LITERAL = 0x200
 FLAG_ASSIGN = 0x400
+FLAG_BEST_EFFORT = 0x800
 
 SCHED_NO, SCHED_YES, SCHED_INVALID = 0, 1, 2
-WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID = -1, -2, -3, -4
+WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID, WCRT_BEST_EFFORT = -1, -2, -3, -4, -5
 ITER_CAP = 1 << 20
 
 _FIELDS = ("task_off", "period", "deadline", "priority", "core",

@@ -23,7 +23,13 @@
  *   - without the LITERAL flag: Lemma 7's jitter J^c_h is 0 for a CPU-only tau_h, and
  *     Lemma 10's same-core term is charged to a CPU-only tau_i too;
  *   - Lemma 4's interleaving-set size is nu_i = N_g - |{h in hpp(i): eta^g_h > 0}| + 1 and
- *     Lemma 1's is N_g - 1 (N_g = number of GPU-using tasks of the taskset).
+ *     Lemma 1's is N_g - 1 (N_g = number of GPU-using tasks of the taskset);
+ *   - with FLAG_BEST_EFFORT a task whose priority value is <= 0 is a best-effort task (Table 4
+ *     prints priority 0 for the two tasks "not assigned real-time priority"; Sec. 7.1 runs
+ *     such tasks "with the lowest priority in the system"): it has no deadline to meet, is
+ *     never analysed (BEST_EFFORT in out_wcrt) and, being below every real-time task, is in
+ *     no hp() or hpp(); it still shares the time-sliced GPU under round robin, so it counts
+ *     in N_g (Lemma 1, Lemma 4).  Under GCAPS it is preempted at once and adds nothing.
  * Parity unpinned: the sentinel convention, the iteration cap and the two repaired forms are
  * not fixed by the paper; the tests pin them only through hand-derived vectors.
  */
@@ -42,6 +48,7 @@ typedef __int128 wide;
 #define POLICY_RR 1
 #define FLAG_BUSY 0x100
 #define FLAG_LITERAL 0x200
+#define FLAG_BEST_EFFORT 0x800
 
 #define SCHED_NO 0
 #define SCHED_YES 1
@@ -50,6 +57,7 @@ typedef __int128 wide;
 #define WCRT_SKIPPED (-2)
 #define WCRT_ITER_LIMIT (-3)
 #define WCRT_INVALID (-4)
+#define WCRT_BEST_EFFORT (-5)
 
 typedef struct {
   int64_t n_tasks, n_csegs, n_gsegs;
@@ -104,6 +112,7 @@ static int analyse_taskset(const oracle_tasksets_t *ts, int64_t t, int policy_fl
   const int policy = policy_flags & 0xff;
   const int busy = (policy_flags & FLAG_BUSY) != 0;
   const int literal = (policy_flags & FLAG_LITERAL) != 0;
+  const int best_effort = (policy_flags & FLAG_BEST_EFFORT) != 0;
 
   int bad = check_taskset(ts, t);
   if (bad) {
@@ -148,6 +157,10 @@ static int analyse_taskset(const oracle_tasksets_t *ts, int64_t t, int policy_fl
   for (int pos = 0; pos < n; ++pos) {
     const int i = order[pos];
     const int64_t k = first + i;
+    if (best_effort && ts->priority[k] <= 0) { /* not a real-time task: nothing to bound */
+      out_wcrt[k] = WCRT_BEST_EFFORT;
+      continue;
+    }
     if (sched != SCHED_YES) {
       out_wcrt[k] = WCRT_SKIPPED;
       continue;
@@ -268,7 +281,7 @@ int oracle_rta_range(const oracle_tasksets_t *ts, int64_t first, int64_t count, 
                      uint8_t *out_sched, oracle_counts_t *counts) {
   const int policy = policy_flags & 0xff;
   if (policy != POLICY_GCAPS && policy != POLICY_RR) return -1;
-  if (policy_flags & ~(0xff | FLAG_BUSY | FLAG_LITERAL)) return -1;
+  if (policy_flags & ~(0xff | FLAG_BUSY | FLAG_LITERAL | FLAG_BEST_EFFORT)) return -1;
   if (ovh < 0 || ovh > MAX_TIME) return -1;
   if (policy == POLICY_RR && (L < 1 || L > MAX_TIME)) return -1;
   oracle_counts_t local = {0, 0, 0};

@@ -10,7 +10,7 @@ from paper_2406_05221_b200.taskgen import TasksetBatch
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
 POLICY = {"gcaps": 0, "rr": 1}
-BUSY, LITERAL = 0x100, 0x200
+BUSY, LITERAL, BEST_EFFORT = 0x100, 0x200, 0x800
 ALL_MODES = [0, BUSY, LITERAL, BUSY | LITERAL, 1, 1 | BUSY, 1 | LITERAL, 1 | BUSY | LITERAL]
 
 
@@ -31,7 +31,8 @@ def parse_vectors(name):
                                   cseg=cseg, gseg=gseg))
             elif tok[0] == "case":
                 flags = POLICY[kv["policy"]] | (BUSY if kv["busy"] == "1" else 0) | (
-                    LITERAL if kv["literal"] == "1" else 0)
+                    LITERAL if kv["literal"] == "1" else 0) | (
+                    BEST_EFFORT if kv.get("be", "0") == "1" else 0)
                 cases.append(dict(name=tok[1], policy=flags, L=int(kv["L"]), ovh=int(kv["ovh"]),
                                   expect=[int(x) for x in kv["expect"].split(",")]))
     return tasks, cases
