@@ -44,12 +44,23 @@ extern "C" {
  *                       as 0 for a CPU-only tau_h (a task without GPU segments never suspends);
  *                       (b) GCAPS busy-waiting, Lemma 10: the busy-wait G^{e*}_h of a same-core
  *                       GPU-using tau_h is charged to tau_i also when tau_i is CPU-only.
+ *   GCAPS_RTA_BEST_EFFORT  tasks whose priority value is <= 0 are best-effort tasks: tasks
+ *                       without a real-time priority that run below every real-time task (the
+ *                       last experiment of Sec. 7.1; Table 4 prints priority 0 for them).  Such a
+ *                       task has no deadline to meet: it is not analysed, gets
+ *                       GCAPS_WCRT_BEST_EFFORT and never makes a taskset unschedulable.  It
+ *                       interferes with no real-time task on the CPU, nor on the GPU under GCAPS
+ *                       (it is preempted at once); under round robin it takes its turns on the
+ *                       time-sliced GPU like any GPU-using task, i.e. it counts in the number of
+ *                       GPU-using tasks of Lemma 1 and Lemma 4.  Real-time tasks then need
+ *                       priorities > 0.  Without the flag a value <= 0 is an ordinary priority.
  */
 #define GCAPS_POLICY_GCAPS 0
 #define GCAPS_POLICY_RR 1
 #define GCAPS_RTA_BUSY 0x100
 #define GCAPS_RTA_LITERAL 0x200
 #define GCAPS_RTA_ASSIGN 0x400 /* only for gcaps_rta_gpu_priority_batch: search the GPU priorities */
+#define GCAPS_RTA_BEST_EFFORT 0x800 /* not accepted by gcaps_rta_gpu_priority_batch */
 
 /* ---- values written to out_sched[t] --------------------------------------------------------- */
 #define GCAPS_SCHED_NO 0      /* some task's bound exceeds its deadline (or hit ITER_LIMIT)      */
@@ -61,6 +72,7 @@ extern "C" {
 #define GCAPS_WCRT_SKIPPED (-2)    /* every task after the first MISS / ITER_LIMIT in that order */
 #define GCAPS_WCRT_ITER_LIMIT (-3) /* GCAPS_RTA_ITER_CAP sweeps without convergence or miss      */
 #define GCAPS_WCRT_INVALID (-4)    /* task of an INVALID taskset (when its slot is addressable)  */
+#define GCAPS_WCRT_BEST_EFFORT (-5) /* best-effort task (GCAPS_RTA_BEST_EFFORT): not analysed    */
 
 /* ---- return codes ---------------------------------------------------------------------------- */
 #define GCAPS_OK 0

@@ -20,9 +20,10 @@ POLICY_RR = 1
 BUSY = 0x100
 LITERAL = 0x200
 ASSIGN = 0x400
+BEST_EFFORT = 0x800
 
 SCHED_NO, SCHED_YES, SCHED_INVALID = 0, 1, 2
-WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID = -1, -2, -3, -4
+WCRT_MISS, WCRT_SKIPPED, WCRT_ITER_LIMIT, WCRT_INVALID, WCRT_BEST_EFFORT = -1, -2, -3, -4, -5
 MAX_TASKS = 256
 MAX_TIME = 1 << 40
 

@@ -214,6 +214,7 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
   const int policy = p.policy & 0xff;
   const bool busy = (p.policy & GCAPS_RTA_BUSY) != 0;
   const bool literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
+  const bool best_effort = (p.policy & GCAPS_RTA_BEST_EFFORT) != 0;
   const u64 L = (u64)p.L, ovh = (u64)p.ovh;
 
   const i64 a = p.task_off[t] - p.task_base, b = p.task_off[t + 1] - p.task_base;
@@ -277,7 +278,8 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
     s.Star[rank] = policy == GCAPS_POLICY_GCAPS ? 2 * ovh * (u64)eta : sat_mul(L + ovh, slices);
     s.core[rank] = (int)p.core[k];
     s.eta[rank] = eta;
-    s.ord[rank] = (unsigned short)i;
+    // a best-effort task (flag set, priority <= 0) ranks behind every real-time task; bit 15
+    s.ord[rank] = (unsigned short)(i | ((best_effort && pi <= 0) ? 0x8000 : 0));
   }
   bad = group_or<LPT>(bad, mask);
   const int n_gpu = group_sum_int<LPT>(n_gpu_lane, mask);  // N_g
@@ -288,12 +290,14 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
     if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
     return;
   }
-  for (int i = lane; i < n; i += LPT) s.prio_out[i] = GCAPS_WCRT_SKIPPED;
+  for (int i = lane; i < n; i += LPT)
+    s.prio_out[i] = (best_effort && s.prio_out[i] <= 0) ? GCAPS_WCRT_BEST_EFFORT : GCAPS_WCRT_SKIPPED;
   __syncwarp(mask);
 
   // ---- iterate: tasks in decreasing priority ---------------------------------------------------
   int sched = GCAPS_SCHED_YES;
   for (int pos = 0; pos < n; ++pos) {
+    if (s.ord[pos] & 0x8000) break;  // only best-effort tasks from here on: nothing to bound
     const u64 Di = s.D[pos];
     const int core_i = s.core[pos];
     const bool gi = s.eta[pos] > 0;
@@ -363,11 +367,11 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
     if (verdict == 0) {
       if (lane == 0) {
         s.R[pos] = R;
-        s.prio_out[s.ord[pos]] = (i64)R;
+        s.prio_out[s.ord[pos] & 0x7fff] = (i64)R;
       }
       __syncwarp(mask);
     } else {
-      if (lane == 0) s.prio_out[s.ord[pos]] = verdict;
+      if (lane == 0) s.prio_out[s.ord[pos] & 0x7fff] = verdict;
       sched = GCAPS_SCHED_NO;
       break;
     }
@@ -586,12 +590,14 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   constexpr int BG = 1;
   constexpr bool kGcaps = MODE < 2;
   const bool literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
+  const bool best_effort = (p.policy & GCAPS_RTA_BEST_EFFORT) != 0;
   uint4 *info = reinterpret_cast<uint4 *>(buf + Lay::kInfo);
   u32 *Q0 = buf + Lay::kQ0, *Q1 = buf + Lay::kQ1;
 
   // ---- stage: per-task scalars, lane = position; rank ----------------------------------------
   u32 T[SLOTS];
   int rank[SLOTS], c0[SLOTS], g0[SLOTS];
+  bool be[SLOTS];  // best-effort task: flag set and priority <= 0
   bool ok = true;
   int Nc, Ng;
   i64 cfirst, gfirst;
@@ -625,6 +631,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       D[s] = (u32)d64[s];
       core[s] = (u32)c64[s];
       prio[s] = v ? (int)pr[s] : (int)0x80000000;
+      be[s] = best_effort && v && pr[s] <= 0;
       c0[s] = v ? (int)rc : Nc;
       g0[s] = v ? (int)rg : Ng;
       high |= v ? h : 0u;
@@ -830,14 +837,14 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   for (int s = 0; s < SLOTS; ++s) {
     if (lane + LPT * s < n) {
       *(reinterpret_cast<uint2 *>(&info[rank[s]]) + 1) =
-          make_uint2(base[s], (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u));
+          make_uint2(base[s], (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u) | (be[s] ? 0x20000u : 0u));
       xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], S[s]);
     }
   }
   __syncwarp(gmask);
   // by rank from here on: period - 1, C+G^m, G^e, S, the two weights of the analysis' pairs
   u32 Tm1[SLOTS], Ar[SLOTS], Ger[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS], core[SLOTS];
-  bool gpu[SLOTS];
+  bool gpu[SLOTS], be_r[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + LPT * s;
@@ -846,6 +853,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     const u32 Sr = x.w;
     Tm1[s] = x.x - 1, Ar[s] = x.y, Ger[s] = x.z;
     core[s] = f.y, pos_of[s] = f.w & 0xffffu, gpu[s] = (f.w & 0x10000u) != 0;
+    be_r[s] = (f.w & 0x20000u) != 0;
     if (MODE == 0) {
       Wa[s] = Ar[s] + (gpu[s] ? Sr : 0u);    // Lemma 15: C_h, or C_h + G^{m*}_h
       Wb[s] = gpu[s] ? Ger[s] + Sr : 0u;     // Lemma 13, other cores: G^{e*}_h
@@ -866,6 +874,10 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   int verdict = 0;
   for (int pos = 0; pos < n; ++pos) {
     const uint4 f = info[pos];
+    if (f.w & 0x20000u) {  // only best-effort tasks from here on (they rank last): nothing to bound
+      n_done = pos;
+      break;
+    }
     const u32 Di = f.x, core_i = f.y, base_i = f.z;
     const bool gi = (f.w & 0x10000u) != 0;
     const int smax = (pos - 1) >> kLog;  // -1 for the first task: nothing interferes
@@ -961,7 +973,8 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     for (int s = 0; s < SLOTS; ++s) {
       const int r = lane + LPT * s;
       if (r < n && r >= n_done)
-        out_wcrt[a + pos_of[s]] = r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED;
+        out_wcrt[a + pos_of[s]] = be_r[s] ? (i64)GCAPS_WCRT_BEST_EFFORT
+                                          : (r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED);
     }
   }
   if (lane == 0) out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
@@ -1433,7 +1446,8 @@ int check_args(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy, int64
   if (!ts || n_tasksets < 0 || n_tasksets > 0x7fffffffLL) return GCAPS_ERR_INVALID_ARG;
   const int pol = policy & 0xff;
   if (pol != GCAPS_POLICY_GCAPS && pol != GCAPS_POLICY_RR) return GCAPS_ERR_INVALID_ARG;
-  if (policy & ~(0xff | GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL)) return GCAPS_ERR_INVALID_ARG;
+  if (policy & ~(0xff | GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL | GCAPS_RTA_BEST_EFFORT))
+    return GCAPS_ERR_INVALID_ARG;
   if (ovh < 0 || ovh > GCAPS_RTA_MAX_TIME) return GCAPS_ERR_INVALID_ARG;
   if (pol == GCAPS_POLICY_RR && (L < 1 || L > GCAPS_RTA_MAX_TIME)) return GCAPS_ERR_INVALID_ARG;
   if (ts->n_tasks < 0 || ts->n_csegs < 0 || ts->n_gsegs < 0) return GCAPS_ERR_INVALID_ARG;
