@@ -251,7 +251,7 @@ def main():
             if events is not None:
                 events[k].record(stream)
             if args.mode == "assign" and k == 1:
-                binding.rta_gpu_priority(ts, binding.ASSIGN, ovh, None, stream=stream)
+                binding.rta_gpu_priority(ts, binding.ASSIGN, ovh, None, workspace=workspace, stream=stream)
             elif args.mode == "sweep" and k == 0:
                 binding.rta_sweep(ts, sweep_policy, [a for a, _ in pairs], [b for _, b in pairs],
                                   out_wcrt=sweep_wcrt, out_sched=sweep_sched, workspace=workspace,
@@ -379,7 +379,7 @@ def main():
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": args.steps * (len(policies) * LAUNCHES_PER_CALL if args.mode == "policies"
                                           else (1 + len(pairs)) * LAUNCHES_PER_CALL if args.mode == "sweep"
-                                          else LAUNCHES_PER_CALL + 1),
+                                          else 2 * LAUNCHES_PER_CALL),
             "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
         }
         print(json.dumps(line))

@@ -174,7 +174,9 @@ int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int pol
  * segments of every task (Sec. 5.3 "Separate Priority for GPU Segments", Sec. 6.4 "Analysis for
  * GPU Priority Assignment").  hp(tau_i) of Lemmas 10, 11 and 13 becomes the set of tasks with a
  * higher GPU-segment priority, hpp(tau_i) keeps its meaning (same core, higher CPU priority),
- * and every jitter uses D_h in place of R_h, so each task is analysed on its own.
+ * and every jitter uses D_h in place of R_h, so each task is analysed on its own:
+ * J^c_h = D_h - (C_h + G^m_h), J^g_h = D_h - G^e_h (0 where the task's own execution exceeds
+ * its deadline).
  *
  *   flags               GCAPS_RTA_BUSY, GCAPS_RTA_LITERAL (as for gcaps_rta_batch), GCAPS_RTA_ASSIGN
  *   runlist_update_us   epsilon (Def. 2), 0..MAX_TIME
@@ -193,13 +195,15 @@ int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int pol
  *   out_wcrt            DEVICE, [ts->n_tasks]: the task's bound, GCAPS_WCRT_MISS (also: never
  *                       placed) or GCAPS_WCRT_ITER_LIMIT; nothing is SKIPPED here
  *   out_sched           DEVICE, [n_tasksets]: 1 if every task has a bound within its deadline
+ *   workspace           DEVICE scratch as for gcaps_rta_batch (gcaps_rta_workspace_bytes() bytes,
+ *                       256-byte aligned): the size-binned launch plan
  *
- * Asynchronous on `stream`, no workspace, no allocation.  Same return codes as gcaps_rta_batch.
+ * Asynchronous on `stream`, no allocation.  Same return codes as gcaps_rta_batch.
  */
 int gcaps_rta_gpu_priority_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int flags,
                                  int64_t runlist_update_us, const int64_t *gpu_priority,
                                  int64_t *out_gpu_priority, int64_t *out_wcrt, uint8_t *out_sched,
-                                 void *stream);
+                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * gcaps_rta_batch_host_multi -- gcaps_rta_batch_host for several analyses of the same batch (the

@@ -20,7 +20,8 @@
  * segments take part in the assignment like any other; every task gets its own outcome (bound,
  * MISS or ITER_LIMIT; nothing is SKIPPED because nothing depends on an earlier task); when the
  * assignment fails at some level the tasks still unassigned get MISS and GPU priority 0; given
- * GPU priorities that break the same-core rule make the taskset INVALID.
+ * GPU priorities that break the same-core rule make the taskset INVALID; a jitter D_h - (C_h +
+ * G^m_h) or D_h - G^e_h that would be negative (a task that cannot meet its own deadline) is 0.
  */
 #include <stdint.h>
 
@@ -98,8 +99,13 @@ static int64_t bound_of(const model_t *m, int i, const unsigned char *above_gpu,
       const int hp_gpu = above_gpu[h] && !hpp; /* hp(tau_i) of Sec. 6.4 without hpp(tau_i) */
       const int gh = m->eta[h] > 0;
       const wide star = 2 * (wide)eps * m->eta[h];
-      const wide Jc = m->D[h] - (m->C[h] + m->Gm[h]); /* Sec. 6.4: D_h in place of R_h */
-      const wide Jg = m->D[h] - m->Ge[h];
+      /* Sec. 6.4: D_h in place of R_h.  The substitution presumes R_h <= D_h; a task whose own
+       * execution already exceeds its deadline has no such slack, and its jitter is taken as 0
+       * (that task gets MISS on its own account, so the taskset fails either way). */
+      wide Jc = m->D[h] - (m->C[h] + m->Gm[h]);
+      wide Jg = m->D[h] - m->Ge[h];
+      if (Jc < 0) Jc = 0;
+      if (Jg < 0) Jg = 0;
       if (!busy) {
         if (hpp && !gh) next += ceil_div(R, m->T[h]) * m->C[h];                              /* Lemma 15 */
         if (hpp && gh) next += ceil_div(R + Jc, m->T[h]) * (m->C[h] + m->Gm[h] + star);      /* Lemma 15 */

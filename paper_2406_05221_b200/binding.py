@@ -85,7 +85,8 @@ def load_library(path: Optional[str] = None):
         lib.gcaps_rta_batch_host_multi.restype = ctypes.c_int
         lib.gcaps_rta_gpu_priority_batch.argtypes = [
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_void_p,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+            ctypes.c_void_p]
         lib.gcaps_rta_gpu_priority_batch.restype = ctypes.c_int
         lib.gcaps_rta_sweep_batch.argtypes = [
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int, _p64, _p64,
@@ -216,7 +217,7 @@ def rta_batch_static(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, 
 
 
 def rta_gpu_priority(ts: DeviceTasksets, flags: int = 0, overhead_us: int = 0, gpu_priority=None,
-                     stream=None):
+                     workspace=None, stream=None):
     """gcaps_rta_gpu_priority_batch: GCAPS with separate GPU-segment priorities.  ``gpu_priority``
     is an int64 CUDA tensor per task, or None together with ``ASSIGN`` in ``flags`` to search the
     priorities.  Returns ``(out_wcrt, out_sched, out_gpu_priority)`` CUDA tensors."""
@@ -227,11 +228,14 @@ def rta_gpu_priority(ts: DeviceTasksets, flags: int = 0, overhead_us: int = 0, g
         out_wcrt = torch.full((ts.n_tasks,), WCRT_INVALID, dtype=torch.int64, device=dev)
         out_sched = torch.full((max(ts.n_tasksets, 0),), SCHED_INVALID, dtype=torch.uint8, device=dev)
         out_gp = torch.zeros(ts.n_tasks, dtype=torch.int64, device=dev)
+        if workspace is None:
+            workspace = torch.empty(max(workspace_bytes(ts.n_tasksets), 256), dtype=torch.uint8, device=dev)
         st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_gpu_priority_batch(
             ctypes.byref(ts.c), ts.n_tasksets, flags, overhead_us,
             gpu_priority.data_ptr() if gpu_priority is not None else None, out_gp.data_ptr(),
-            out_wcrt.data_ptr(), out_sched.data_ptr(), st.cuda_stream)
+            out_wcrt.data_ptr(), out_sched.data_ptr(), workspace.data_ptr(), workspace.numel(),
+            st.cuda_stream)
     _check(rc)
     return out_wcrt, out_sched, out_gp
 

@@ -7,11 +7,13 @@ import sys
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CUDA_SRC = os.path.join(_HERE, "csrc", "gcaps_rta.cu")
+CUDA_SRCS = [CUDA_SRC, os.path.join(_HERE, "csrc", "gcaps_gpu_priority.cu")]
+CUDA_DEPS = CUDA_SRCS + [os.path.join(_HERE, "csrc", "rta_common.cuh")]
 CUDA_LIB = os.path.join(_HERE, "libgcaps_rta.so")
 HEADER = os.path.join(os.path.dirname(_HERE), "include", "gcaps_rta.h")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-shared", "-Xcompiler", "-fPIC"]
+              "-shared", "-Xcompiler", "-fPIC", "--threads", "2"]
 
 
 def _nvcc() -> str:
@@ -25,16 +27,16 @@ def cuda_lib_is_stale() -> bool:
     if not os.path.exists(CUDA_LIB):
         return True
     m = os.path.getmtime(CUDA_LIB)
-    return m < os.path.getmtime(CUDA_SRC) or m < os.path.getmtime(HEADER)
+    return any(m < os.path.getmtime(f) for f in CUDA_DEPS + [HEADER])
 
 
 def build_cuda(force: bool = False, verbose: bool = False) -> str:
-    """Compiles csrc/gcaps_rta.cu for sm_100a into libgcaps_rta.so beside this file."""
+    """Compiles the CUDA sources of csrc/ for sm_100a into libgcaps_rta.so beside this file."""
     if force or cuda_lib_is_stale():
         tmp = CUDA_LIB + ".%d.tmp" % os.getpid()
         if os.path.exists(CUDA_LIB):
             os.remove(CUDA_LIB)  # a failed build must not leave an older library behind
-        cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp, CUDA_SRC]
+        cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + CUDA_SRCS
         subprocess.check_call(cmd)
         os.replace(tmp, CUDA_LIB)
     return CUDA_LIB

@@ -28,72 +28,11 @@
 #include <stdio.h>
 #include <string.h>
 
-#include "../../include/gcaps_rta.h"
+#include "rta_common.cuh"
+
+using namespace gcaps_detail;
 
 namespace {
-
-typedef unsigned long long u64;
-typedef long long i64;
-
-constexpr int kNumBins = 9;
-constexpr int kBinStride = 12;  // counters per plan block and per header array
-typedef unsigned int u32;
-// size bins: at most 8, 16, 24, 32, 64, 96, 128, 192, 256 tasks
-constexpr u32 kFastLimit = 1u << 26;  // fast path: every time of the taskset is below this
-constexpr u32 kFastClamp = 1u << 26;  // ... so a sum clamped here still exceeds every deadline
-constexpr int kBlockThreads = 128;
-constexpr int kPlanItems = 1024;  // tasksets per plan block
-constexpr u64 kClamp = 1ull << 50;  // any quantity >= 2^50 exceeds every deadline (<= 2^40)
-
-struct PlanHeader {
-  unsigned int bin_start[kBinStride];
-  unsigned int bin_count[kBinStride];
-  unsigned int next[kBinStride];  // work counters of the analysis launches
-};
-static_assert(sizeof(PlanHeader) <= 256, "header layout");
-
-struct KParams {
-  const i64 *task_off, *period, *deadline, *priority, *core;
-  const i64 *cseg_off, *cseg_wcet, *gseg_off, *gseg_misc, *gseg_exec;
-  i64 n_tasks, n_csegs, n_gsegs;        // lengths of the arrays the pointers address
-  i64 task_base, cseg_base, gseg_base;  // subtracted from the stored offsets (chunked host path)
-  i64 n_tasksets;
-  int policy;  // GCAPS_POLICY_* | flags
-  i64 L, ovh;
-  // division by L in the 32-bit path: 0 = multiply-high by l_magic then shift, 1 = L is 1,
-  // 2 = L >= 2^26 (every non-empty pure GPU part takes one slice)
-  u32 l_mode, l_magic, l_shift;
-  i64 *out_wcrt;
-  uint8_t *out_sched;
-  PlanHeader *hdr;
-  unsigned int *block_cnt;  // [plan blocks][kBinStride]
-  unsigned int *perm;       // [n_tasksets]
-};
-
-// The (timeslice, overhead) pairs of a fused sweep: one staging and aggregation of a taskset,
-// one analysis per pair.  Passed to the sweep kernels by value.
-struct SweepPoint {
-  i64 L, ovh;
-  u32 l_mode, l_magic, l_shift, pad;  // division by L in the 32-bit path, as in KParams
-};
-struct SweepArgs {
-  int n;        // pairs, 1 .. GCAPS_RTA_MAX_SWEEP
-  i64 max_ovh;  // largest overhead of the sweep
-  SweepPoint q[GCAPS_RTA_MAX_SWEEP];
-};
-
-__device__ __forceinline__ int size_bin(i64 n) {
-  if (n <= 8) return 0;  // also negative / broken ranges: rejected by the analysis kernel
-  if (n <= 16) return 1;
-  if (n <= 24) return 2;
-  if (n <= 32) return 3;
-  if (n <= 64) return 4;
-  if (n <= 96) return 5;
-  if (n <= 128) return 6;
-  if (n <= 192) return 7;
-  if (n <= GCAPS_RTA_MAX_TASKS) return 8;
-  return 0;
-}
 
 // ---------------------------------------------------------------------------------------------
 // plan: counting sort of taskset indices by size bin (histogram per block, scan, scatter)
@@ -160,34 +99,6 @@ __global__ void plan_scatter_kernel(KParams p) {
       p.perm[p.hdr->bin_start[b] + slot] = (unsigned int)t;
     }
   }
-}
-
-// ---------------------------------------------------------------------------------------------
-// exact saturating helpers of the 64-bit path
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ u64 sat_mul(u64 a, u64 b) {  // min(a*b, kClamp)
-  u64 lo = a * b;
-  return (__umul64hi(a, b) != 0 || lo > kClamp) ? kClamp : lo;
-}
-__device__ __forceinline__ u64 ceil_div64(u64 a, u64 b) { return (a + b - 1) / b; }
-
-template <int LPT>
-__device__ __forceinline__ u64 group_sum(u64 v, unsigned int mask) {
-#pragma unroll
-  for (int d = LPT / 2; d >= 1; d >>= 1) v += __shfl_xor_sync(mask, v, d, LPT);
-  return v;
-}
-template <int LPT>
-__device__ __forceinline__ int group_or(int v, unsigned int mask) {
-#pragma unroll
-  for (int d = LPT / 2; d >= 1; d >>= 1) v |= __shfl_xor_sync(mask, v, d, LPT);
-  return v;
-}
-template <int LPT>
-__device__ __forceinline__ int group_sum_int(int v, unsigned int mask) {
-#pragma unroll
-  for (int d = LPT / 2; d >= 1; d >>= 1) v += __shfl_xor_sync(mask, v, d, LPT);
-  return v;
 }
 
 // Shared-memory image of one taskset, indexed by priority rank unless noted.
@@ -386,54 +297,6 @@ __device__ void analyse_taskset(const KParams &p, i64 t, GroupSmem<MAXN> &s, int
 // ---------------------------------------------------------------------------------------------
 // 32-bit fast path
 // ---------------------------------------------------------------------------------------------
-constexpr unsigned int kFull = 0xffffffffu;
-
-__device__ __forceinline__ u32 warp_incl_scan(u32 x, int lane) {
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const u32 y = __shfl_up_sync(kFull, x, d);
-    if (lane >= d) x += y;
-  }
-  return x;
-}
-
-// Reciprocal of a divisor d in [2, 2^26): floor(x / d) = umulhi(x, magic) >> shift for every
-// x < 2^28.  With s = ceil(log2 d) and k = max(28 + s, 32), magic = ceil(2^k / d) < 2^32 and its
-// error magic*d - 2^k < d <= 2^s, so x * error < 2^k and the quotient is exact.
-__host__ __device__ __forceinline__ void make_reciprocal(u32 d, u32 &magic, u32 &shift) {
-#ifdef __CUDA_ARCH__
-  const int s = 32 - __clz((int)(d - 1));
-#else
-  int s = 0;
-  while ((1u << s) < d) ++s;
-#endif
-  const int k = (28 + s) > 32 ? (28 + s) : 32;
-  shift = (u32)(k - 32);
-#ifdef __CUDA_ARCH__
-  // estimate 2^k / d in single precision (off by less than 2^10), correct the estimate once with
-  // the same approximate reciprocal (off by at most 1 then), and finish with integers.  Checked
-  // against the exact quotient for every d in [2, 2^26), also with the reciprocal off by 8 ulp.
-  float inv;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(__uint2float_rn(d)));
-  const u32 q0 = __float2uint_rd(inv * __int_as_float((127 + k) << 23));
-  const i64 rem0 = (i64)(1ull << k) - (i64)((u64)q0 * d);
-  const int c = __float2int_rd(__ll2float_rn(rem0) * inv);
-  u32 q = q0 + (u32)c;
-  i64 rem = rem0 - (i64)c * (i64)d;
-  if (rem < 0) {
-    q -= 1;
-    rem += d;
-  } else if (rem >= (i64)d) {
-    q += 1;
-    rem -= d;
-  }
-  magic = rem == 0 ? q : q + 1;
-#else
-  const u64 two_k = 1ull << k;
-  magic = (u32)((two_k + d - 1) / d);
-#endif
-}
-
 // ---- running sums of a segment array, 128 elements per step ------------------------------------
 // Lane l takes four consecutive elements (two 16-byte loads), so a warp reads 1 KB contiguous.
 // Loads must start on a 16-byte boundary: when the slice starts on an odd element the step begins
@@ -1170,207 +1033,6 @@ rta_big_sweep_kernel(KParams p, int bin, const __grid_constant__ SweepArgs sw) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// separate GPU-segment priorities (Sec. 5.3, Sec. 6.4): one warp per taskset, exact arithmetic
-// ---------------------------------------------------------------------------------------------
-struct GpSmem {  // by position
-  u64 T[GCAPS_RTA_MAX_TASKS], D[GCAPS_RTA_MAX_TASKS];
-  u64 A[GCAPS_RTA_MAX_TASKS];     // C + G^m
-  u64 Ge[GCAPS_RTA_MAX_TASKS];    // G^e
-  u64 Star[GCAPS_RTA_MAX_TASKS];  // 2 * eps * eta^g
-  i64 key[GCAPS_RTA_MAX_TASKS];   // priorities while ranking
-  int core[GCAPS_RTA_MAX_TASKS];
-  int eta[GCAPS_RTA_MAX_TASKS];
-  short cpu_rank[GCAPS_RTA_MAX_TASKS], gpu_rank[GCAPS_RTA_MAX_TASKS];
-  short by_cpu_rank[GCAPS_RTA_MAX_TASKS];  // CPU rank -> position
-  unsigned char above[GCAPS_RTA_MAX_TASKS];  // 1: has a higher GPU priority than the task analysed
-};
-
-// Bound of task i when the tasks flagged in s.above[] have a higher GPU-segment priority: the
-// recurrence of Sec. 6.3 with hp() by GPU priority and D_h in the jitters (Sec. 6.4).  Lanes over
-// the other tasks.  Returns the bound, GCAPS_WCRT_MISS or GCAPS_WCRT_ITER_LIMIT (warp-uniform).
-__device__ i64 gp_bound(const GpSmem &s, int n, int i, bool busy, bool literal, u64 eps, int lane) {
-  const bool gi = s.eta[i] > 0;
-  const u64 base = s.A[i] + s.Ge[i] + s.Star[i] + ((u64)s.eta[i] + 1) * eps;  // C_i + G*_i + B^C_i
-  const u64 Di = s.D[i];
-  const int core_i = s.core[i], rank_i = s.cpu_rank[i];
-  u64 R = base;
-  i64 sweeps = 0;
-  for (;;) {
-    if (R > Di) return GCAPS_WCRT_MISS;
-    if (sweeps >= GCAPS_RTA_ITER_CAP) return GCAPS_WCRT_ITER_LIMIT;
-    sweeps += 1;
-    u64 part = 0;
-    for (int h = lane; h < n; h += 32) {
-      if (h == i) continue;
-      const bool hpp = s.core[h] == core_i && s.cpu_rank[h] < rank_i;
-      const bool hp_gpu = s.above[h] != 0 && !hpp;
-      const bool gh = s.eta[h] > 0;
-      const u64 Th = s.T[h];
-      const u64 Jc = s.D[h] - s.A[h], Jg = s.D[h] - s.Ge[h];
-      u64 term = 0;
-      if (!busy) {
-        if (hpp && !gh) term = sat_mul(ceil_div64(R, Th), s.A[h]);                  // Lemma 15
-        if (hpp && gh) term = sat_mul(ceil_div64(R + Jc, Th), s.A[h] + s.Star[h]);  // Lemma 15
-        if (hpp && gh && gi) term += sat_mul(ceil_div64(R + Jg, Th), s.Ge[h]);      // Lemma 13
-        if (hp_gpu && gh && gi) term = sat_mul(ceil_div64(R + Jg, Th), s.Ge[h] + s.Star[h]);
-      } else {
-        if (hpp) {
-          u64 W = s.A[h];                                          // Lemma 12
-          if (gh && (gi || !literal)) W += s.Ge[h] + s.Star[h];    // Lemma 10
-          term = sat_mul(ceil_div64(R, Th), W);
-        } else if (hp_gpu && gh) {
-          term = sat_mul(ceil_div64(R + Jg, Th), s.Ge[h] + s.Star[h]);  // Lemmas 10, 11
-        }
-      }
-      part += term;
-    }
-    const u64 next = base + group_sum<32>(part, kFull);
-    if (next == R) return (i64)R;
-    R = next;
-  }
-}
-
-struct GpParams {
-  KParams k;
-  const i64 *gpu_prio_in;
-  i64 *gpu_prio_out;
-  int assign;
-};
-
-__global__ void __launch_bounds__(kBlockThreads) gpu_priority_kernel(GpParams g) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const KParams &p = g.k;
-  const int lane = threadIdx.x & 31;
-  GpSmem &s = reinterpret_cast<GpSmem *>(smem_raw)[threadIdx.x >> 5];
-  const i64 t = (i64)blockIdx.x * (kBlockThreads / 32) + (threadIdx.x >> 5);
-  if (t >= p.n_tasksets) return;
-  const bool busy = (p.policy & GCAPS_RTA_BUSY) != 0, literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
-  const u64 eps = (u64)p.ovh;
-  const i64 a = p.task_off[t], b = p.task_off[t + 1];
-  if (a < 0 || b < a || b > p.n_tasks || b - a > GCAPS_RTA_MAX_TASKS) {
-    if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
-    return;
-  }
-  const int n = (int)(b - a);
-  // ---- stage, validate, aggregate (task model of Sec. 4) ----------------------------------
-  int bad = 0;
-  for (int i = lane; i < n; i += 32) {
-    const i64 k = a + i;
-    const i64 T = p.period[k], D = p.deadline[k], c = p.core[k];
-    if (T < 1 || T > GCAPS_RTA_MAX_TIME) bad |= GCAPS_BAD_PERIOD;
-    if (D < 1 || D > T) bad |= GCAPS_BAD_DEADLINE;
-    if (c < 0 || c > GCAPS_RTA_MAX_CORE) bad |= GCAPS_BAD_CORE;
-    const i64 c0 = p.cseg_off[k], c1 = p.cseg_off[k + 1], g0 = p.gseg_off[k], g1 = p.gseg_off[k + 1];
-    const bool seg_ok = !(c0 < 0 || c1 < c0 || c1 > p.n_csegs || c1 - c0 > GCAPS_RTA_MAX_SEGMENTS ||
-                          g0 < 0 || g1 < g0 || g1 > p.n_gsegs || g1 - g0 > GCAPS_RTA_MAX_SEGMENTS);
-    u64 C = 0, Gm = 0, Ge = 0;
-    if (seg_ok) {
-      for (i64 j = c0; j < c1; ++j) {
-        const i64 w = p.cseg_wcet[j];
-        if (w < 0 || w > GCAPS_RTA_MAX_TIME) bad |= GCAPS_BAD_WCET;
-        C += (u64)w;
-      }
-      for (i64 j = g0; j < g1; ++j) {
-        const i64 m = p.gseg_misc[j], e = p.gseg_exec[j];
-        if (m < 0 || m > GCAPS_RTA_MAX_TIME || e < 0 || e > GCAPS_RTA_MAX_TIME) bad |= GCAPS_BAD_WCET;
-        Gm += (u64)m, Ge += (u64)e;
-      }
-    } else {
-      bad |= GCAPS_BAD_SEG_RANGE;
-    }
-    const int eta = seg_ok ? (int)(g1 - g0) : 0;
-    s.T[i] = (u64)T, s.D[i] = (u64)D, s.A[i] = C + Gm, s.Ge[i] = Ge;
-    s.Star[i] = 2 * eps * (u64)eta;
-    s.core[i] = (int)c, s.eta[i] = eta;
-    s.key[i] = p.priority[k];
-  }
-  bad = group_or<32>(bad, kFull);
-  __syncwarp();
-  if (bad) {
-    for (int i = lane; i < n; i += 32) {
-      p.out_wcrt[a + i] = GCAPS_WCRT_INVALID;
-      if (g.gpu_prio_out) g.gpu_prio_out[a + i] = 0;
-    }
-    if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
-    return;
-  }
-  for (int i = lane; i < n; i += 32) {  // CPU ranks: larger priority first, ties by position
-    const i64 pi = s.key[i];
-    int r = 0;
-    for (int q = 0; q < n; ++q) r += (s.key[q] > pi || (s.key[q] == pi && q < i)) ? 1 : 0;
-    s.cpu_rank[i] = (short)r;
-    s.by_cpu_rank[r] = (short)i;
-  }
-  __syncwarp();
-  int sched = GCAPS_SCHED_YES;
-  if (!g.assign) {
-    for (int i = lane; i < n; i += 32) s.key[i] = g.gpu_prio_in[a + i];
-    __syncwarp();
-    for (int i = lane; i < n; i += 32) {
-      const i64 pi = s.key[i];
-      int r = 0;
-      for (int q = 0; q < n; ++q) r += (s.key[q] > pi || (s.key[q] == pi && q < i)) ? 1 : 0;
-      s.gpu_rank[i] = (short)r;
-    }
-    __syncwarp();
-    int broken = 0;  // same core: the GPU order must equal the CPU order (Sec. 5.3)
-    for (int i = lane; i < n; i += 32)
-      for (int q = 0; q < n; ++q)
-        if (s.core[i] == s.core[q] && s.cpu_rank[q] < s.cpu_rank[i] && s.gpu_rank[q] > s.gpu_rank[i]) broken = 1;
-    if (group_or<32>(broken, kFull)) {
-      for (int i = lane; i < n; i += 32) p.out_wcrt[a + i] = GCAPS_WCRT_INVALID;
-      if (lane == 0) p.out_sched[t] = GCAPS_SCHED_INVALID;
-      return;
-    }
-    for (int i = 0; i < n; ++i) {
-      for (int q = lane; q < n; q += 32) s.above[q] = s.gpu_rank[q] < s.gpu_rank[i] ? 1 : 0;
-      __syncwarp();
-      const i64 r = gp_bound(s, n, i, busy, literal, eps, lane);
-      if (lane == 0) {
-        p.out_wcrt[a + i] = r;
-        if (g.gpu_prio_out) g.gpu_prio_out[a + i] = g.gpu_prio_in[a + i];
-      }
-      if (r < 0) sched = GCAPS_SCHED_NO;
-      __syncwarp();
-    }
-  } else {
-    // gpu_rank doubles as "unassigned" flag here: -1 while the task has no level yet
-    for (int i = lane; i < n; i += 32) {
-      s.gpu_rank[i] = -1;
-      p.out_wcrt[a + i] = GCAPS_WCRT_MISS;
-      g.gpu_prio_out[a + i] = 0;
-    }
-    __syncwarp();
-    for (int level = 1; level <= n && sched == GCAPS_SCHED_YES; ++level) {
-      bool placed = false;
-      for (int want = n - 1; want >= 0 && !placed; --want) {  // lowest CPU priority first
-        const int c = s.by_cpu_rank[want];
-        if (s.gpu_rank[c] >= 0) continue;
-        int lower = 0;  // an unassigned task of lower CPU priority on the same core bars c
-        for (int q = lane; q < n; q += 32)
-          if (q != c && s.gpu_rank[q] < 0 && s.core[q] == s.core[c] && s.cpu_rank[q] > s.cpu_rank[c]) lower = 1;
-        if (group_or<32>(lower, kFull)) continue;
-        for (int q = lane; q < n; q += 32) s.above[q] = (s.gpu_rank[q] < 0 && q != c) ? 1 : 0;
-        __syncwarp();
-        const i64 r = gp_bound(s, n, c, busy, literal, eps, lane);
-        __syncwarp();
-        if (r >= 0) {
-          placed = true;
-          if (lane == 0) {
-            s.gpu_rank[c] = (short)level;
-            p.out_wcrt[a + c] = r;
-            g.gpu_prio_out[a + c] = (i64)level;
-          }
-          __syncwarp();
-        }
-      }
-      if (!placed) sched = GCAPS_SCHED_NO;
-    }
-  }
-  if (lane == 0) p.out_sched[t] = (uint8_t)sched;
-}
-
-// ---------------------------------------------------------------------------------------------
 // validation kernel: one thread per taskset
 // ---------------------------------------------------------------------------------------------
 __global__ void validate_kernel(KParams p, int32_t *out_err) {
@@ -1403,16 +1065,20 @@ __global__ void validate_kernel(KParams p, int32_t *out_err) {
   out_err[t] = bad;
 }
 
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+size_t plan_blocks(int64_t n_tasksets) { return (size_t)((n_tasksets + kPlanItems - 1) / kPlanItems); }
+
+}  // namespace
+
 // ---------------------------------------------------------------------------------------------
-// host side
+// host side shared with the other translation units of the library
 // ---------------------------------------------------------------------------------------------
+namespace gcaps_detail {
+
 thread_local int g_last_cuda_error = 0;
 
-struct DeviceInfo {
-  int sm_count;
-  int ok;  // 1 = usable sm_100 device, -1 = not usable
-};
-DeviceInfo g_dev[64];
+static DeviceInfo g_dev[64];
 
 int device_info(DeviceInfo *out) {
   int dev = 0;
@@ -1437,10 +1103,6 @@ int device_info(DeviceInfo *out) {
   *out = g_dev[dev];
   return GCAPS_OK;
 }
-
-size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
-size_t plan_blocks(int64_t n_tasksets) { return (size_t)((n_tasksets + kPlanItems - 1) / kPlanItems); }
 
 int check_args(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy, int64_t L, int64_t ovh) {
   if (!ts || n_tasksets < 0 || n_tasksets > 0x7fffffffLL) return GCAPS_ERR_INVALID_ARG;
@@ -1494,29 +1156,24 @@ void fill_params(KParams *p, const gcaps_tasksets_t *ts, int64_t n_tasksets, int
   p->out_sched = out_sched;
 }
 
-// Launches `kernel` (a persistent kernel of kBlockThreads threads needing `smem` bytes) with as
-// many blocks as the device keeps resident, but never more than the batch could feed.
-template <typename... Args>
-cudaError_t launch_persistent(void (*kernel)(Args...), int *blocks_per_sm, size_t smem, long long want,
-                              int sm_count, cudaStream_t st, Args... args) {
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  dev &= 63;
-  if (blocks_per_sm[dev] == 0) {  // first use on this device
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    int per_sm = 1;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlockThreads, smem);
-    if (e != cudaSuccess) return e;
-    blocks_per_sm[dev] = per_sm < 1 ? 1 : per_sm;
-  }
-  long long grid = (long long)sm_count * blocks_per_sm[dev];
-  if (grid > want) grid = want;
-  if (grid < 1) grid = 1;
-  kernel<<<(unsigned int)grid, kBlockThreads, smem, st>>>(args...);
-  return cudaGetLastError();
+int enqueue_plan(KParams &p, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+  const size_t need = gcaps_rta_workspace_bytes(p.n_tasksets);
+  if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255u))
+    return GCAPS_ERR_WORKSPACE;
+  unsigned char *w = (unsigned char *)workspace;
+  const size_t nb = plan_blocks(p.n_tasksets);
+  p.hdr = (PlanHeader *)w;
+  p.block_cnt = (unsigned int *)(w + 256);
+  p.perm = (unsigned int *)(w + 256 + align_up(nb * kBinStride * sizeof(unsigned int), 256));
+  plan_count_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
+  plan_scan_kernel<<<1, 32 * kNumBins, 0, st>>>(p, (unsigned int)nb);
+  plan_scatter_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
+  return GCAPS_OK;
 }
+
+}  // namespace gcaps_detail
+
+namespace {
 
 template <int SLOTS, int MODE>
 cudaError_t launch_big(const KParams &p, int bin, int sm_count, cudaStream_t st) {
@@ -1570,17 +1227,8 @@ cudaError_t launch_all_bins_sweep(const KParams &p, const SweepArgs &sw, int sm_
 int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_count, cudaStream_t st,
                   const SweepArgs *sw = nullptr) {
   if (p.n_tasksets == 0) return GCAPS_OK;
-  const size_t need = gcaps_rta_workspace_bytes(p.n_tasksets);
-  if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255u))
-    return GCAPS_ERR_WORKSPACE;
-  unsigned char *w = (unsigned char *)workspace;
-  const size_t nb = plan_blocks(p.n_tasksets);
-  p.hdr = (PlanHeader *)w;
-  p.block_cnt = (unsigned int *)(w + 256);
-  p.perm = (unsigned int *)(w + 256 + align_up(nb * kBinStride * sizeof(unsigned int), 256));
-  plan_count_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
-  plan_scan_kernel<<<1, 32 * kNumBins, 0, st>>>(p, (unsigned int)nb);
-  plan_scatter_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
+  const int rc = enqueue_plan(p, workspace, workspace_bytes, st);
+  if (rc != GCAPS_OK) return rc;
   cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) {
     const bool rr = (p.policy & 0xff) == GCAPS_POLICY_RR, busy = (p.policy & GCAPS_RTA_BUSY) != 0;
@@ -1710,48 +1358,6 @@ int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int p
   // analysis kernels of this call read.
   return enqueue_batch(p, g_static_scratch_ptr[dev], (size_t)GCAPS_RTA_STATIC_SCRATCH_BYTES,
                        di.sm_count, (cudaStream_t)stream);
-}
-
-int gcaps_rta_gpu_priority_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int flags,
-                                 int64_t runlist_update_us, const int64_t *gpu_priority,
-                                 int64_t *out_gpu_priority, int64_t *out_wcrt, uint8_t *out_sched,
-                                 void *stream) {
-  if (flags & ~(GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL | GCAPS_RTA_ASSIGN)) return GCAPS_ERR_INVALID_ARG;
-  int rc = check_args(ts, n_tasksets, GCAPS_POLICY_GCAPS | (flags & (GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL)),
-                      1, runlist_update_us);
-  if (rc != GCAPS_OK) return rc;
-  const bool assign = (flags & GCAPS_RTA_ASSIGN) != 0;
-  if (n_tasksets == 0) return GCAPS_OK;
-  if (!out_sched || (ts->n_tasks > 0 && (!out_wcrt || (assign ? !out_gpu_priority : !gpu_priority))))
-    return GCAPS_ERR_INVALID_ARG;
-  DeviceInfo di;
-  rc = device_info(&di);
-  if (rc != GCAPS_OK) return rc;
-  GpParams g;
-  fill_params(&g.k, ts, n_tasksets, GCAPS_POLICY_GCAPS | (flags & (GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL)), 1,
-              runlist_update_us, out_wcrt, out_sched);
-  g.gpu_prio_in = (const i64 *)gpu_priority;
-  g.gpu_prio_out = (i64 *)out_gpu_priority;
-  g.assign = assign ? 1 : 0;
-  constexpr int kWarps = kBlockThreads / 32;
-  const size_t smem = sizeof(GpSmem) * kWarps;
-  static bool attr_done[64] = {false};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e == cudaSuccess && !attr_done[dev & 63]) {
-    e = cudaFuncSetAttribute(gpu_priority_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess) attr_done[dev & 63] = true;
-  }
-  if (e == cudaSuccess) {
-    const unsigned int grid = (unsigned int)((n_tasksets + kWarps - 1) / kWarps);
-    gpu_priority_kernel<<<grid, kBlockThreads, smem, (cudaStream_t)stream>>>(g);
-    e = cudaGetLastError();
-  }
-  if (e != cudaSuccess) {
-    g_last_cuda_error = (int)e;
-    return GCAPS_ERR_CUDA;
-  }
-  return GCAPS_OK;
 }
 
 int gcaps_rta_validate(const gcaps_tasksets_t *ts, int64_t n_tasksets, int32_t *out_err,

@@ -124,3 +124,18 @@ def test_bounds_hold_in_simulation_with_assigned_priorities():
                 resp, unf = sim.simulate(b, 0, off, 0, busy, 1, 2 * hyper + max(off) + 1, gpu_priority=gp)
                 assert (resp <= w).all() and (unf <= w).all(), (ts, gp, off, w, resp)
     assert checked > 300
+
+
+def test_jitter_of_a_task_that_cannot_meet_its_own_deadline_is_zero():
+    """Sec. 6.4 puts D_h where Sec. 6.3 has R_h, which presumes R_h <= D_h.  tau_h here needs
+    C + G^m = 35 > D = 20: J^c_h is taken as 0, not -15.  By hand for the lower task (eps = 0):
+    R = 6 + ceil(R/40)*35 + ceil((R+17)/40)*3 -> 6, 44, 82, 120, 123, 158, 161, 196, 199, 199."""
+    sets = [[dict(T=40, D=20, prio=2, core=0, cseg=[30], gseg=[(5, 3)]),
+             dict(T=400, D=400, prio=1, core=0, cseg=[3], gseg=[(1, 2)])]]
+    b = batch_of(sets)
+    wcrt, sched, _ = rta.analyse_gpu_priority(b, 0, 0, gpu_priority=np.array([2, 1]))
+    assert wcrt.tolist() == [rta.WCRT_MISS, 199] and sched.tolist() == [0]
+    # far below zero: still no negative term (base + 35 per job of tau_h at least)
+    sets[0][0]["cseg"] = [3000]
+    wcrt, _, _ = rta.analyse_gpu_priority(batch_of(sets), 0, 0, gpu_priority=np.array([2, 1]))
+    assert wcrt.tolist() == [rta.WCRT_MISS, rta.WCRT_MISS]
