@@ -460,7 +460,6 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   // ---- stage: per-task scalars, lane = position; rank ----------------------------------------
   u32 T[SLOTS];
   int rank[SLOTS], c0[SLOTS], g0[SLOTS];
-  bool be[SLOTS];  // best-effort task: flag set and priority <= 0
   bool ok = true;
   int Nc, Ng;
   i64 cfirst, gfirst;
@@ -494,7 +493,6 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       D[s] = (u32)d64[s];
       core[s] = (u32)c64[s];
       prio[s] = v ? (int)pr[s] : (int)0x80000000;
-      be[s] = best_effort && v && pr[s] <= 0;
       c0[s] = v ? (int)rc : Nc;
       g0[s] = v ? (int)rg : Ng;
       high |= v ? h : 0u;
@@ -540,6 +538,18 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
         }
         rank[s] = i < n ? r : MAXN;
       }
+    }
+    // best-effort tasks (flag set, priority <= 0) rank behind every real-time task: the ranks
+    // from n_rt on are theirs
+    // (kept in a spare word in front of Q0's guard entry until the recurrence starts)
+    {
+      int n_rt = n;
+      if (best_effort) {
+#pragma unroll
+        for (int s = 0; s < SLOTS; ++s)
+          n_rt -= __popc(__ballot_sync(gmask, lane + LPT * s < n && prio[s] <= 0));
+      }
+      if (lane == 0) Q0[-2] = (u32)n_rt;
     }
     // what every lane must know about the task of a given rank (base and GPU flag follow)
 #pragma unroll
@@ -700,14 +710,14 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   for (int s = 0; s < SLOTS; ++s) {
     if (lane + LPT * s < n) {
       *(reinterpret_cast<uint2 *>(&info[rank[s]]) + 1) =
-          make_uint2(base[s], (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u) | (be[s] ? 0x20000u : 0u));
+          make_uint2(base[s], (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u));
       xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], S[s]);
     }
   }
   __syncwarp(gmask);
   // by rank from here on: period - 1, C+G^m, G^e, S, the two weights of the analysis' pairs
   u32 Tm1[SLOTS], Ar[SLOTS], Ger[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS], core[SLOTS];
-  bool gpu[SLOTS], be_r[SLOTS];
+  bool gpu[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + LPT * s;
@@ -716,7 +726,6 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     const u32 Sr = x.w;
     Tm1[s] = x.x - 1, Ar[s] = x.y, Ger[s] = x.z;
     core[s] = f.y, pos_of[s] = f.w & 0xffffu, gpu[s] = (f.w & 0x10000u) != 0;
-    be_r[s] = (f.w & 0x20000u) != 0;
     if (MODE == 0) {
       Wa[s] = Ar[s] + (gpu[s] ? Sr : 0u);    // Lemma 15: C_h, or C_h + G^{m*}_h
       Wb[s] = gpu[s] ? Ger[s] + Sr : 0u;     // Lemma 13, other cores: G^{e*}_h
@@ -733,14 +742,11 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   u32 Jc[SLOTS], Jg[SLOTS];               // jitters with T_h - 1 folded in (ceiling)
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Tm1[s];
-  int n_done = n;
+  const int n_rt = (int)Q0[-2];  // real-time tasks: the ranks that are analysed
+  int n_done = n_rt;
   int verdict = 0;
-  for (int pos = 0; pos < n; ++pos) {
+  for (int pos = 0; pos < n_rt; ++pos) {
     const uint4 f = info[pos];
-    if (f.w & 0x20000u) {  // only best-effort tasks from here on (they rank last): nothing to bound
-      n_done = pos;
-      break;
-    }
     const u32 Di = f.x, core_i = f.y, base_i = f.z;
     const bool gi = (f.w & 0x10000u) != 0;
     const int smax = (pos - 1) >> kLog;  // -1 for the first task: nothing interferes
@@ -836,7 +842,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     for (int s = 0; s < SLOTS; ++s) {
       const int r = lane + LPT * s;
       if (r < n && r >= n_done)
-        out_wcrt[a + pos_of[s]] = be_r[s] ? (i64)GCAPS_WCRT_BEST_EFFORT
+        out_wcrt[a + pos_of[s]] = r >= n_rt ? (i64)GCAPS_WCRT_BEST_EFFORT
                                           : (r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED);
     }
   }
