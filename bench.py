@@ -39,58 +39,11 @@ LAUNCHES_PER_CALL = 9
 # grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
 # the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "de335bca07754e68950253b73e2f4809f8d0244a3f70fc907aaed1ba700fbd57",
+    "source_sha256": "40666923b4df87b626a15993f173a82490dcf20f8e7ce21a42103b36dca5c544",
     "workload": "large",
-    "bytes_per_taskset": {"gcaps": (1247450000 + 83256832) / 131072.0,
-                          "rr": (1245200000 + 81212160) / 131072.0},
+    "bytes_per_taskset": {"gcaps": (1248194000 + 84010496) / 131072.0,
+                          "rr": (1247363000 + 83190272) / 131072.0},
 }
-
-
-def captured_traffic(workload_name, policy_name, tasksets):
-    """DRAM traffic of one analysis launch, or None if the capture does not apply any more."""
-    import hashlib
-    src = os.path.join(ROOT, "paper_2406_05221_b200", "csrc", "gcaps_rta.cu")
-    try:
-        with open(src, "rb") as fh:
-            digest = hashlib.sha256(fh.read()).hexdigest()
-    except OSError:
-        return None
-    if digest != CAPTURED_TRAFFIC["source_sha256"] or workload_name != CAPTURED_TRAFFIC["workload"]:
-        return None
-    per_taskset = CAPTURED_TRAFFIC["bytes_per_taskset"].get(policy_name)
-    return per_taskset * tasksets if per_taskset is not None else None
-
-
-def measured_peaks():
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    try:
-        with open(path) as fh:
-            d = json.load(fh)
-        return float(d["hbm_gbs"]), "measured"
-    except Exception:
-        return FALLBACK_HBM_GBS, "fallback"
-
-
-class ClockSampler:
-    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while a region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
-
-    def __init__(self, gpu_id: str):
-        self.gpu_id, self.proc = gpu_id, None
-
-    def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", self.gpu_id, "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except Exception:
-            self.proc = None
-
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
         time.sleep(0.15)
