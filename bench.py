@@ -44,6 +44,62 @@ CAPTURED_TRAFFIC = {
     "bytes_per_taskset": {"gcaps": (1248194000 + 84010496) / 131072.0,
                           "rr": (1247363000 + 83190272) / 131072.0},
 }
+
+
+def kernel_source_digest():
+    """sha256 over the sources of the analysis kernel (gcaps_rta.cu and the header it shares)."""
+    import hashlib
+    h = hashlib.sha256()
+    try:
+        for name in ("gcaps_rta.cu", "rta_common.cuh"):
+            with open(os.path.join(ROOT, "paper_2406_05221_b200", "csrc", name), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return h.hexdigest()
+
+
+def captured_traffic(workload_name, policy_name, tasksets):
+    """DRAM traffic of one analysis launch, or None if the capture does not apply any more."""
+    digest = kernel_source_digest()
+    if digest is None:
+        return None
+    if digest != CAPTURED_TRAFFIC["source_sha256"] or workload_name != CAPTURED_TRAFFIC["workload"]:
+        return None
+    per_taskset = CAPTURED_TRAFFIC["bytes_per_taskset"].get(policy_name)
+    return per_taskset * tasksets if per_taskset is not None else None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id, self.proc = gpu_id, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.gpu_id, "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
         time.sleep(0.15)
