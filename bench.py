@@ -129,14 +129,14 @@ class ClockSampler:
         return out
 
 
-def oracle_sample(workload, first, count, budget_s, chunk=50_000):
+def oracle_sample(workload, first, count, budget_s, chunk=50_000, stream=0):
     """Times the CPU oracle (as it stands, one thread) on tasksets first.. of the workload, both
     policies per taskset, stopping after ``count`` tasksets or ``budget_s`` seconds."""
     from oracle import rta
     done, spent, terms, sweeps, started = 0, 0.0, [0, 0], [0, 0], [0, 0]
     while done < count and spent < budget_s:
         n = min(chunk, count - done)
-        batch = workload.generate(first + done, n)
+        batch = workload.generate(first + done, n, stream=stream)
         t0 = time.perf_counter()
         for k, policy in enumerate((rta.POLICY_GCAPS, rta.POLICY_RR)):
             _, _, c = rta.analyse(batch, policy, workload.timeslice_us, workload.overhead_us)
@@ -188,6 +188,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--ref-sample", type=int, default=100_000)
+    ap.add_argument("--on-device-inputs", action="store_true",
+                    help="generate the tasksets on the GPU (integer-only generator) instead of on the "
+                         "host; reports the generation time in config.generation")
     ap.add_argument("--mode", default="policies", choices=["policies", "assign", "sweep"],
                     help="policies: GCAPS + RR calls per step (the benchmark); assign: the GCAPS call "
                          "followed by the GPU-priority search of the paper's Sec. 5.3 on the same batch; "
@@ -228,8 +231,30 @@ def main():
         pinned.append(t)
         return t.numpy()[:n]
 
-    batch = workload.generate(first, count, stream=args.stream, alloc=alloc)
-    ts = binding.DeviceTasksets.from_host(batch, dev)
+    generation = None
+    if args.on_device_inputs:
+        # the inputs never exist on the host; the host twin of the same stream is only needed by
+        # the end-to-end and CPU-baseline legs, which are switched off here
+        args.no_e2e = args.no_cpu_baseline = True
+        generation = {}
+        binding.generate_device(workload.streams[args.stream], first, min(count, 1000), dev)  # warm-up
+        ts = binding.generate_device(workload.streams[args.stream], first, count, dev, timing=generation)
+        generation["tasksets_per_s"] = count / ((generation["count_ms"] + generation["fill_ms"]) * 1e-3)
+        generation["generator"] = "integer-only, on device (gcaps_gen_count + gcaps_gen_fill)"
+
+        class _Sizes:   # what the report needs of a host batch
+            def input_bytes(self):
+                return ts.input_bytes()
+
+            def output_bytes(self):
+                return 8 * ts.n_tasks + ts.n_tasksets
+
+            def checksum(self):
+                return None
+        batch = _Sizes()
+    else:
+        batch = workload.generate(first, count, stream=args.stream, alloc=alloc)
+        ts = binding.DeviceTasksets.from_host(batch, dev)
     out_wcrt = torch.empty(ts.n_tasks, dtype=torch.int64, device=dev)
     out_sched = torch.empty(ts.n_tasksets, dtype=torch.uint8, device=dev)
     workspace = torch.empty(max(256, binding.workspace_bytes(ts.n_tasksets)), dtype=torch.uint8, device=dev)
@@ -355,7 +380,7 @@ def main():
                 "frac_per_policy": {nm: bytes_per_call / (ms * 1e-3) / 1e9 / peak
                                     for nm, ms in zip(names, per_policy_ms)}}
         if world == 1 and not args.no_cpu_baseline and args.mode == "policies":
-            r = oracle_sample(workload, first, count, args.cpu_budget)
+            r = oracle_sample(workload, first, count, args.cpu_budget, stream=args.stream)
             cpu = {"value": r["tasksets"] / r["seconds"], "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": "first %d tasksets of the workload, both policies, %.1f s, generation excluded"
                              % (r["tasksets"], r["seconds"]),
@@ -380,7 +405,7 @@ def main():
                        "tasks": ts.n_tasks, "policies": names, "mode": "self-suspension",
                        "timeslice_us": L, "overhead_us": ovh,
                        "analyses_per_taskset_per_step": len(pairs) if pairs else len(policies),
-                       "sweep_pairs": pairs,
+                       "sweep_pairs": pairs, "generation": generation,
                        "l2": "inputs (%.2f GB per call) against a 126 MB L2; no flush between steps"
                              % (batch.input_bytes() / 1e9),
                        "schedulable_fraction_last_policy": sched_frac,

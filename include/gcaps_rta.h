@@ -274,6 +274,60 @@ int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int p
                            int64_t timeslice_us, int64_t ctx_switch_overhead_us,
                            int64_t *out_wcrt, uint8_t *out_sched, void *stream);
 
+/*
+ * On-device taskset generation.  The paper's experiments analyse randomly generated tasksets
+ * (Sec. 7.1, Table 3: tasks per CPU, utilisation per CPU split over its tasks, period, number of
+ * GPU segments, segment parameters, rate-monotonic priorities, worst-fit-decreasing allocation).
+ * These two calls produce such tasksets directly in device memory, in the layout of
+ * gcaps_tasksets_t, so that a large sweep never moves its inputs over the host link.  The
+ * generator is integer-only (fixed point with 32 fractional bits, SplitMix64 as a counter-based
+ * random source): taskset `index` of a stream is a pure function of (seed, stream, index), and
+ * the host generator of the package's taskgen module yields the same bits.
+ *
+ * gcaps_gen_params_t: all "Q32" fields are value * 2^32.
+ */
+typedef struct gcaps_gen_params {
+  uint64_t seed, stream;
+  int32_t cores_lo, cores_hi;    /* CPUs per taskset, uniform, at most 64                       */
+  int32_t tpc_lo, tpc_hi;        /* tasks per CPU, uniform; at most 256 tasks per taskset       */
+  uint64_t util_lo, util_hi;     /* utilisation per CPU, Q32, uniform, below 1                  */
+  uint64_t log2_lo, log2_hi;     /* log2 of the period range (us), Q32: periods are log-uniform */
+  uint64_t log2_hi0;             /* harmonic tasksets: upper end of log2 of the base period     */
+  int64_t period_lo, period_hi;  /* us, clamp of every period; period_hi <= 2^30                */
+  uint64_t harmonic;             /* Q32 share of tasksets whose periods are P0 * 2^k, k <= 10   */
+  uint64_t gpu_frac;             /* Q32 share of GPU-using tasks (gpu_mode 0)                   */
+  uint64_t ratio_lo, ratio_hi;   /* G_i / (C_i + G_i), Q32, uniform, below 1                    */
+  int32_t gpu_mode;              /* 0: exactly round(gpu_frac * n) GPU-using tasks with seg_lo ..
+                                    seg_hi segments; 1: every task draws seg_lo .. seg_hi       */
+  int32_t seg_lo, seg_hi;        /* GPU segments per task, at most 16                           */
+  int32_t wfd;                   /* 1: worst-fit-decreasing re-allocation of tasks to CPUs      */
+} gcaps_gen_params_t;
+
+/* Scratch of gcaps_gen_count / gcaps_gen_fill for `count` tasksets (host computation). */
+size_t gcaps_gen_workspace_bytes(int64_t count);
+
+/*
+ * gcaps_gen_count -- sizes of tasksets first .. first+count-1 of the stream: writes their
+ * offsets into `workspace` (kept for gcaps_gen_fill) and the three array lengths n_tasks,
+ * n_csegs, n_gsegs to out_totals (DEVICE, 3 x int64; read them back to size the arrays).
+ * workspace: DEVICE, gcaps_gen_workspace_bytes(count) bytes, 256-byte aligned.  Asynchronous on
+ * `stream`; GCAPS_OK or a GCAPS_ERR_* (parameters outside the limits stated above:
+ * GCAPS_ERR_INVALID_ARG).
+ */
+int gcaps_gen_count(const gcaps_gen_params_t *params, int64_t first, int64_t count,
+                    int64_t *out_totals, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * gcaps_gen_fill -- writes the tasksets whose offsets gcaps_gen_count (same params, first, count,
+ * workspace) left in `workspace` into the DEVICE arrays of `ts` (ts->n_tasks, n_csegs, n_gsegs
+ * state how many elements the arrays hold; a taskset that would not fit is left out and
+ * GCAPS_ERR_TOO_LARGE is NOT reported asynchronously -- size the arrays from out_totals).
+ * D_i = T_i.  Asynchronous on `stream`.
+ */
+int gcaps_gen_fill(const gcaps_gen_params_t *params, int64_t first, int64_t count,
+                   const gcaps_tasksets_t *ts, void *workspace, size_t workspace_bytes,
+                   void *stream);
+
 /* Frees the staging memory gcaps_rta_batch_host keeps on the current device. */
 void gcaps_rta_release_host(void);
 

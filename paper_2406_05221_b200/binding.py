@@ -13,7 +13,7 @@ from typing import Dict, Optional, Tuple
 import numpy as np
 
 from . import build as _build
-from .taskgen import ARRAY_FIELDS, TasksetBatch
+from .taskgen import ARRAY_FIELDS, GenParams, IntParams, TasksetBatch
 
 POLICY_GCAPS = 0
 POLICY_RR = 1
@@ -34,7 +34,8 @@ MAX_SWEEP = 32
 EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host",
            "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
            "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static",
-           "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch", "gcaps_rta_sweep_batch")
+           "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch", "gcaps_rta_sweep_batch",
+           "gcaps_gen_workspace_bytes", "gcaps_gen_count", "gcaps_gen_fill")
 
 _p64 = ctypes.POINTER(ctypes.c_int64)
 
@@ -92,6 +93,15 @@ def load_library(path: Optional[str] = None):
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int, _p64, _p64,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         lib.gcaps_rta_sweep_batch.restype = ctypes.c_int
+        lib.gcaps_gen_workspace_bytes.argtypes = [ctypes.c_int64]
+        lib.gcaps_gen_workspace_bytes.restype = ctypes.c_size_t
+        lib.gcaps_gen_count.argtypes = [ctypes.POINTER(IntParams), ctypes.c_int64, ctypes.c_int64,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        lib.gcaps_gen_count.restype = ctypes.c_int
+        lib.gcaps_gen_fill.argtypes = [ctypes.POINTER(IntParams), ctypes.c_int64, ctypes.c_int64,
+                                       ctypes.POINTER(CTasksets), ctypes.c_void_p, ctypes.c_size_t,
+                                       ctypes.c_void_p]
+        lib.gcaps_gen_fill.restype = ctypes.c_int
         lib.gcaps_rta_release_host.argtypes = []
         lib.gcaps_rta_release_host.restype = None
         lib.gcaps_rta_validate.argtypes = [ctypes.POINTER(CTasksets), ctypes.c_int64,
@@ -238,6 +248,46 @@ def rta_gpu_priority(ts: DeviceTasksets, flags: int = 0, overhead_us: int = 0, g
             st.cuda_stream)
     _check(rc)
     return out_wcrt, out_sched, out_gp
+
+
+def generate_device(params: GenParams, first: int, count: int, device="cuda:0", stream=None,
+                    timing=None) -> DeviceTasksets:
+    """gcaps_gen_count + gcaps_gen_fill: tasksets ``first .. first+count-1`` of the stream, made
+    on the device by the integer-only generator (the same tasksets as
+    ``taskgen.generate(params, first, count, integer=True)``).  One 24-byte read-back of the array
+    lengths sits between the two calls; nothing else crosses the host link.  ``timing``, if a
+    dict, receives the device time of both calls in ms."""
+    import torch
+    lib = load_library()
+    dev = torch.device(device)
+    cp = params.int_params()
+    with torch.cuda.device(dev):
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        ws = torch.empty(max(int(lib.gcaps_gen_workspace_bytes(count)), 256), dtype=torch.uint8, device=dev)
+        totals = torch.zeros(3, dtype=torch.int64, device=dev)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if timing is not None else None
+        if ev:
+            ev[0].record(st)
+        _check(lib.gcaps_gen_count(ctypes.byref(cp), first, count, totals.data_ptr(), ws.data_ptr(),
+                                   ws.numel(), st.cuda_stream))
+        if ev:
+            ev[1].record(st)
+        n_tasks, n_c, n_g = (int(x) for x in totals.cpu().tolist())
+        sizes = {"task_off": max(count, 0) + 1, "period": n_tasks, "deadline": n_tasks,
+                 "priority": n_tasks, "core": n_tasks, "cseg_off": n_tasks + 1, "cseg_wcet": n_c,
+                 "gseg_off": n_tasks + 1, "gseg_misc": n_g, "gseg_exec": n_g}
+        t = {f: torch.zeros(sizes[f], dtype=torch.int64, device=dev) for f in ARRAY_FIELDS}
+        ts = DeviceTasksets(t)
+        if ev:
+            ev[2].record(st)
+        _check(lib.gcaps_gen_fill(ctypes.byref(cp), first, count, ctypes.byref(ts.c), ws.data_ptr(),
+                                  ws.numel(), st.cuda_stream))
+        if ev:
+            ev[3].record(st)
+            torch.cuda.synchronize(dev)
+            timing["count_ms"] = ev[0].elapsed_time(ev[1])
+            timing["fill_ms"] = ev[2].elapsed_time(ev[3])
+    return ts
 
 
 def rta_validate(ts: DeviceTasksets, stream=None):

@@ -290,3 +290,66 @@ void tg_fill(const tg_params_t *p, int64_t first, int64_t count, const int64_t *
 
 int tg_max_tasks(void) { return TG_MAX_TASKS; }
 size_t tg_params_size(void) { return sizeof(tg_params_t); }
+
+/* ---------------------------------------------------------------------------------------------
+ * The integer-only generator (igen.h) on the host: the same two passes as above.  Its output is
+ * bit-identical to what the CUDA library's on-device generator writes for the same parameters.
+ * ------------------------------------------------------------------------------------------- */
+#include "igen.h"
+
+void ig_sizes(const igen_params_t *p, int64_t first, int64_t count, int64_t *counts) {
+#pragma omp parallel
+  {
+    igen_state_t *s = (igen_state_t *)malloc(sizeof(igen_state_t));
+#pragma omp for schedule(static)
+    for (int64_t t = 0; t < count; ++t) {
+      igen_begin(p, (uint64_t)(first + t), s);
+      counts[3 * t + 0] = s->n;
+      counts[3 * t + 1] = s->n_csegs;
+      counts[3 * t + 2] = s->n_gsegs;
+    }
+    free(s);
+  }
+}
+
+void ig_fill(const igen_params_t *p, int64_t first, int64_t count, const int64_t *starts,
+             int64_t *task_off, int64_t *period, int64_t *deadline, int64_t *priority,
+             int64_t *core, int64_t *cseg_off, int64_t *cseg_wcet, int64_t *gseg_off,
+             int64_t *gseg_misc, int64_t *gseg_exec) {
+#pragma omp parallel
+  {
+    igen_state_t *s = (igen_state_t *)malloc(sizeof(igen_state_t));
+#pragma omp for schedule(static)
+    for (int64_t t = 0; t < count; ++t) {
+      igen_begin(p, (uint64_t)(first + t), s);
+      int64_t k0 = starts[3 * t + 0], c0 = starts[3 * t + 1], g0 = starts[3 * t + 2];
+      task_off[t] = k0;
+      for (int i = 0; i < s->n; ++i) {
+        int64_t cs[IGEN_MAX_SEGS + 1], gm[IGEN_MAX_SEGS], ge[IGEN_MAX_SEGS];
+        igen_segments(s, i, cs, gm, ge);
+        period[k0 + i] = s->T[i];
+        deadline[k0 + i] = s->T[i];
+        priority[k0 + i] = s->prio[i];
+        core[k0 + i] = s->core[i];
+        cseg_off[k0 + i] = c0;
+        gseg_off[k0 + i] = g0;
+        for (int j = 0; j <= s->eta[i]; ++j) cseg_wcet[c0 + j] = cs[j];
+        for (int j = 0; j < s->eta[i]; ++j) {
+          gseg_misc[g0 + j] = gm[j];
+          gseg_exec[g0 + j] = ge[j];
+        }
+        c0 += s->eta[i] + 1;
+        g0 += s->eta[i];
+      }
+      if (t == count - 1) {
+        task_off[count] = k0 + s->n;
+        cseg_off[k0 + s->n] = c0;
+        gseg_off[k0 + s->n] = g0;
+      }
+    }
+    free(s);
+  }
+}
+
+size_t ig_params_size(void) { return sizeof(igen_params_t); }
+uint64_t ig_exp2(uint64_t y) { return igen_exp2(y); }

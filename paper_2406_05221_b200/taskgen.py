@@ -22,6 +22,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "csrc", "taskgen.c")
+_IGEN_H = os.path.join(_HERE, "csrc", "igen.h")
 _LIB = os.path.join(_HERE, "_taskgen.so")
 _lock = threading.Lock()
 _lib = None
@@ -35,7 +36,8 @@ ARRAY_FIELDS = (
 def build_taskgen(force: bool = False) -> str:
     """Compiles csrc/taskgen.c into _taskgen.so beside this file (gcc, OpenMP)."""
     with _lock:
-        if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(
+                os.path.getmtime(_SRC), os.path.getmtime(_IGEN_H)):
             tmp = _LIB + ".%d.tmp" % os.getpid()
             subprocess.check_call(
                 ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
@@ -59,11 +61,35 @@ class _Params(ctypes.Structure):
     ]
 
 
+class IntParams(ctypes.Structure):
+    """Mirror of ``igen_params_t`` (csrc/igen.h) and of ``gcaps_gen_params_t`` (gcaps_rta.h)."""
+    _fields_ = [
+        ("seed", ctypes.c_uint64), ("stream", ctypes.c_uint64),
+        ("cores_lo", ctypes.c_int32), ("cores_hi", ctypes.c_int32),
+        ("tpc_lo", ctypes.c_int32), ("tpc_hi", ctypes.c_int32),
+        ("util_lo", ctypes.c_uint64), ("util_hi", ctypes.c_uint64),
+        ("log2_lo", ctypes.c_uint64), ("log2_hi", ctypes.c_uint64), ("log2_hi0", ctypes.c_uint64),
+        ("period_lo", ctypes.c_int64), ("period_hi", ctypes.c_int64),
+        ("harmonic", ctypes.c_uint64), ("gpu_frac", ctypes.c_uint64),
+        ("ratio_lo", ctypes.c_uint64), ("ratio_hi", ctypes.c_uint64),
+        ("gpu_mode", ctypes.c_int32), ("seg_lo", ctypes.c_int32), ("seg_hi", ctypes.c_int32),
+        ("wfd", ctypes.c_int32),
+    ]
+
+
 def _load():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(build_taskgen())
         p64 = ctypes.POINTER(ctypes.c_int64)
+        lib.ig_sizes.argtypes = [ctypes.POINTER(IntParams), ctypes.c_int64, ctypes.c_int64, p64]
+        lib.ig_sizes.restype = None
+        lib.ig_fill.argtypes = [ctypes.POINTER(IntParams), ctypes.c_int64, ctypes.c_int64, p64] + [p64] * 10
+        lib.ig_fill.restype = None
+        lib.ig_params_size.restype = ctypes.c_size_t
+        assert lib.ig_params_size() == ctypes.sizeof(IntParams)
+        lib.ig_exp2.argtypes = [ctypes.c_uint64]
+        lib.ig_exp2.restype = ctypes.c_uint64
         lib.tg_sizes.argtypes = [ctypes.POINTER(_Params), ctypes.c_int64, ctypes.c_int64, p64]
         lib.tg_sizes.restype = None
         lib.tg_fill.argtypes = [ctypes.POINTER(_Params), ctypes.c_int64, ctypes.c_int64, p64] + [p64] * 10
@@ -98,6 +124,22 @@ class GenParams:
             self.period_us[0], self.period_us[1], self.harmonic_frac,
             self.gpu_mode, self.gpu_frac, self.gpu_segments[0], self.gpu_segments[1],
             self.gpu_ratio[0], self.gpu_ratio[1], 1 if self.wfd else 0, 0)
+
+    def int_params(self) -> "IntParams":
+        """The same ranges for the integer-only generator: fixed point with 32 fractional bits,
+        period range as log2 (rounded here, once, on the host: both the host and the device
+        generator receive these integers)."""
+        import math
+        lo, hi = float(self.period_us[0]), float(self.period_us[1])
+        hi0 = min(lo * 100.0, hi)
+        return IntParams(
+            self.seed, self.stream, self.cores[0], self.cores[1],
+            self.tasks_per_core[0], self.tasks_per_core[1],
+            q32(self.util_per_core[0]), q32(self.util_per_core[1]),
+            q32(math.log2(lo)), q32(math.log2(hi)), q32(math.log2(hi0)),
+            int(lo), int(hi), q32(self.harmonic_frac), q32(self.gpu_frac),
+            q32(self.gpu_ratio[0]), q32(self.gpu_ratio[1]),
+            self.gpu_mode, self.gpu_segments[0], self.gpu_segments[1], 1 if self.wfd else 0)
 
 
 @dataclasses.dataclass
@@ -239,21 +281,30 @@ def _ranges(start: np.ndarray, length: np.ndarray) -> np.ndarray:
     return np.cumsum(out)
 
 
+def q32(x: float) -> int:
+    """x as a fixed-point number with 32 fractional bits."""
+    return int(round(x * 4294967296.0))
+
+
 def generate(params: GenParams, first: int, count: int, threads: Optional[int] = None,
-             alloc=None) -> TasksetBatch:
+             alloc=None, integer: bool = False) -> TasksetBatch:
     """Tasksets ``first .. first+count-1`` of the stream described by ``params``.
 
-    ``alloc(n)`` may supply the int64 output arrays (e.g. views of page-locked memory)."""
+    ``alloc(n)`` may supply the int64 output arrays (e.g. views of page-locked memory).
+    ``integer=True`` uses the integer-only generator (csrc/igen.h), whose tasksets the CUDA
+    library can also produce on the device, bit for bit; it is a different stream of tasksets
+    with the same ranges and distributions."""
     lib = _load()
     if count <= 0:
         return TasksetBatch.from_tasksets([])
     if threads is not None:
         os.environ["OMP_NUM_THREADS"] = str(threads)
-    cp = params._c()
+    cp = params.int_params() if integer else params._c()
+    sizes_fn, fill_fn = (lib.ig_sizes, lib.ig_fill) if integer else (lib.tg_sizes, lib.tg_fill)
     counts = np.zeros((count, 3), np.int64)
     p64 = ctypes.POINTER(ctypes.c_int64)
     ptr = lambda a: a.ctypes.data_as(p64)
-    lib.tg_sizes(ctypes.byref(cp), first, count, ptr(counts))
+    sizes_fn(ctypes.byref(cp), first, count, ptr(counts))
     starts = np.zeros((count, 3), np.int64)
     np.cumsum(counts[:-1], axis=0, out=starts[1:])
     n_tasks, n_c, n_g = (int(x) for x in counts.sum(axis=0))
@@ -263,7 +314,7 @@ def generate(params: GenParams, first: int, count: int, threads: Optional[int] =
              "core": n_tasks, "cseg_off": n_tasks + 1, "cseg_wcet": n_c, "gseg_off": n_tasks + 1,
              "gseg_misc": n_g, "gseg_exec": n_g}
     arr = {f: alloc(sizes[f]) for f in ARRAY_FIELDS}
-    lib.tg_fill(ctypes.byref(cp), first, count, ptr(starts), *[ptr(arr[f]) for f in ARRAY_FIELDS])
+    fill_fn(ctypes.byref(cp), first, count, ptr(starts), *[ptr(arr[f]) for f in ARRAY_FIELDS])
     return TasksetBatch(**arr)
 
 
@@ -281,10 +332,10 @@ class Workload:
     note: str = ""
 
     def generate(self, first: int = 0, count: Optional[int] = None, stream: int = 0,
-                 alloc=None) -> TasksetBatch:
+                 alloc=None, integer: bool = False) -> TasksetBatch:
         if count is None:
             count = self.n_tasksets - first
-        return generate(self.streams[stream], first, count, alloc=alloc)
+        return generate(self.streams[stream], first, count, alloc=alloc, integer=integer)
 
 
 def _workloads() -> Dict[str, Workload]:

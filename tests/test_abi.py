@@ -13,7 +13,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "gcaps_rta.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(gcaps_rta_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(gcaps_(?:rta|gen)_[a-z_]+)\s*\(", text)))
 
 
 @pytest.fixture(scope="module")
@@ -34,6 +34,7 @@ def test_host_only_entry_points(lib):
     assert binding.workspace_bytes(0) == 0 and binding.workspace_bytes(-5) == 0
     small, big = binding.workspace_bytes(1), binding.workspace_bytes(1_000_000)
     assert small >= 4 and big >= 4 * 1_000_000 and big % 256 == 0
+    assert lib.gcaps_gen_workspace_bytes(0) == 0 and lib.gcaps_gen_workspace_bytes(1000) % 256 == 0
     for code in (0, -1, -2, -3, -4, -99):
         assert lib.gcaps_rta_strerror(code)
 
