@@ -2,7 +2,8 @@
 """Throughput benchmark of the batched response-time analysis (tasksets analysed per second).
 
 A step is one pass of the whole hot path over one batch of synthetic tasksets: the GCAPS
-analysis and the round-robin analysis of every taskset of the batch (two library calls).  The
+analysis and the round-robin analysis of every taskset of the batch (two gcaps_rta_batch calls;
+`--fused`: one gcaps_rta_multi_batch call that reads every taskset once).  The
 default workload is the 1,000,000-taskset configuration (8 cores x 10 tasks per taskset).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
@@ -188,6 +189,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--ref-sample", type=int, default=100_000)
+    ap.add_argument("--fused", action="store_true",
+                    help="one gcaps_rta_multi_batch call per step (every taskset read once, analysed "
+                         "under both policies) instead of one gcaps_rta_batch call per policy")
     ap.add_argument("--on-device-inputs", action="store_true",
                     help="generate the tasksets on the GPU (integer-only generator) instead of on the "
                          "host; reports the generation time in config.generation")
@@ -261,6 +265,14 @@ def main():
     policies = [p for p in (binding.POLICY_GCAPS, binding.POLICY_RR)
                 if ("gcaps", "rr")[p] in workload.policies]
     names = [("gcaps", "rr")[p] for p in policies]
+    host_policies = list(policies)   # the end-to-end leg
+    analyses_per_step = len(policies)
+    fused = args.mode == "policies" and len(policies) == 2 and args.fused
+    if fused:
+        # one call analyses every taskset under GCAPS and under round robin (self-suspension)
+        policies, names = ["fused"], ["gcaps+rr"]
+        multi_wcrt = torch.empty((1, 2, ts.n_tasks), dtype=torch.int64, device=dev)
+        multi_sched = torch.empty((1, 2, ts.n_tasksets), dtype=torch.uint8, device=dev)
     L, ovh = workload.timeslice_us, workload.overhead_us
     stream = torch.cuda.current_stream(dev)
 
@@ -286,6 +298,10 @@ def main():
                 events[k].record(stream)
             if args.mode == "assign" and k == 1:
                 binding.rta_gpu_priority(ts, binding.ASSIGN, ovh, None, workspace=workspace, stream=stream)
+            elif fused:
+                binding.rta_multi(ts, binding.GCAPS_SUSPEND | binding.RR_SUSPEND, [L], [ovh],
+                                  out_wcrt=multi_wcrt, out_sched=multi_sched, workspace=workspace,
+                                  stream=stream)
             elif args.mode == "sweep" and k == 0:
                 binding.rta_sweep(ts, sweep_policy, [a for a, _ in pairs], [b for _, b in pairs],
                                   out_wcrt=sweep_wcrt, out_sched=sweep_sched, workspace=workspace,
@@ -326,7 +342,7 @@ def main():
     total_ms = ev[0][0].elapsed_time(ev[-1][-1])
     per_policy_ms = [statistics.mean(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(len(policies))]
     best_policy_ms = [min(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(len(policies))]
-    flags = sweep_sched[0] if args.mode == "sweep" else out_sched
+    flags = sweep_sched[0] if args.mode == "sweep" else (multi_sched[0, 1] if fused else out_sched)
     sched_frac = float((flags == 1).float().mean().item()) if count else 0.0
     total_ms = sharding.reduce_scalars([total_ms], "max", dev)[0]
     ms_per_step = total_ms / args.steps
@@ -338,22 +354,22 @@ def main():
     e2e = None
     if not args.no_e2e:
         host_wcrt = [torch.empty(max(ts.n_tasks, 1), dtype=torch.int64, pin_memory=True).numpy()[:ts.n_tasks]
-                     for _ in policies]
+                     for _ in host_policies]
         host_sched = [torch.empty(max(ts.n_tasksets, 1), dtype=torch.uint8, pin_memory=True).numpy()[:ts.n_tasksets]
-                      for _ in policies]
+                      for _ in host_policies]
         arrays = batch.arrays()
         # warm-up: staging buffers get allocated here
-        binding.rta_batch_host_multi(arrays, policies, L, ovh, host_wcrt, host_sched)
+        binding.rta_batch_host_multi(arrays, host_policies, L, ovh, host_wcrt, host_sched)
         barrier()
         t0 = time.perf_counter()
         for _ in range(args.e2e_steps):
-            binding.rta_batch_host_multi(arrays, policies, L, ovh, host_wcrt, host_sched)
+            binding.rta_batch_host_multi(arrays, host_policies, L, ovh, host_wcrt, host_sched)
         barrier()
         dt = time.perf_counter() - t0
         dt = sharding.reduce_scalars([dt], "max", dev)[0]
         e2e = {"value": world * count * args.e2e_steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": batch.input_bytes(),
-               "d2h_bytes_per_step": len(policies) * batch.output_bytes(),
+               "d2h_bytes_per_step": len(host_policies) * batch.output_bytes(),
                "steps": args.e2e_steps, "ms_per_step": 1e3 * dt / args.e2e_steps,
                "api": "gcaps_rta_batch_host_multi, page-locked host arrays, one copy in, both policies"}
         binding.release_host()
@@ -363,6 +379,8 @@ def main():
     bytes_per_call = batch.input_bytes() + batch.output_bytes()
     if args.mode == "sweep":  # inputs once, outputs once per pair
         bytes_per_call = batch.input_bytes() + len(pairs) * batch.output_bytes()
+    if fused:                 # inputs once, outputs once per analysis
+        bytes_per_call = batch.input_bytes() + 2 * batch.output_bytes()
     peak, peak_kind = measured_peaks()
     roof = None
     if rank == 0:
@@ -373,7 +391,7 @@ def main():
                 "traffic": captured_traffic(workload.name, names[dom], count),
                 "peak_kind": peak_kind,
                 "kernel": "analysis kernel of the %s call (the call's plan kernels are inside the timing)"
-                          % names[dom].upper(),
+                          % names[dom].upper() + (": both analyses of a taskset in one launch" if fused else ""),
                 "algorithmic_bytes_per_launch": bytes_per_call,
                 "ms_per_launch": dict(zip(names, per_policy_ms)),
                 "best_ms_per_launch": dict(zip(names, best_policy_ms)),
@@ -388,8 +406,8 @@ def main():
             # which roofline binds: algorithmic integer work against algorithmic bytes
             n_tasks_per_set = ts.n_tasks / max(1, ts.n_tasksets)
             t_mem = bytes_per_call / (peak * 1e9)
-            pol_idx = policies[dom]
-            t_alu = count * (K_TERM * r["terms"][pol_idx] / r["tasksets"] + K_SETUP * n_tasks_per_set) / ALU_PEAK_LANEOPS
+            terms = sum(r["terms"]) if fused else r["terms"][policies[dom]]
+            t_alu = count * (K_TERM * terms / r["tasksets"] + K_SETUP * n_tasks_per_set) / ALU_PEAK_LANEOPS
             roof["model_ms"] = {"hbm": 1e3 * t_mem, "alu": 1e3 * t_alu}
             if t_alu > t_mem:
                 ops = t_alu * ALU_PEAK_LANEOPS
@@ -404,7 +422,8 @@ def main():
             "config": {"workload": workload.name, "note": workload.note, "tasksets_per_gpu": count,
                        "tasks": ts.n_tasks, "policies": names, "mode": "self-suspension",
                        "timeslice_us": L, "overhead_us": ovh,
-                       "analyses_per_taskset_per_step": len(pairs) if pairs else len(policies),
+                       "analyses_per_taskset_per_step": len(pairs) if pairs else analyses_per_step,
+                       "calls_per_step": len(policies),
                        "sweep_pairs": pairs, "generation": generation,
                        "l2": "inputs (%.2f GB per call) against a 126 MB L2; no flush between steps"
                              % (batch.input_bytes() / 1e9),

@@ -243,6 +243,32 @@ int gcaps_rta_sweep_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int po
                           size_t workspace_bytes, void *stream);
 
 /*
+ * gcaps_rta_multi_batch -- several analyses of one device-resident batch in a single pass.  The
+ * paper's experiments put every generated taskset through the GCAPS analysis and through the
+ * analysis of the default round-robin driver, in both waiting modes (Sec. 7.1; Sec. 6.2 and 6.3
+ * each give a busy-waiting and a self-suspension lemma set).  Here a taskset is read, ordered
+ * and aggregated once and then goes through the recurrence of gcaps_rta_batch once per requested
+ * analysis and per (timeslice, overhead) pair; the two self-suspension analyses run in one
+ * launch, the two busy-waiting ones in another.  Results are those of separate gcaps_rta_batch
+ * calls.
+ *
+ *   analyses   OR of GCAPS_ANALYSIS_*; `flags`: GCAPS_RTA_LITERAL, GCAPS_RTA_BEST_EFFORT
+ *   n_points, timeslice_us, ctx_switch_overhead_us: as for gcaps_rta_sweep_batch (the overhead of
+ *              a pair is theta for the round-robin analyses and epsilon for the GCAPS ones)
+ *   out_wcrt   DEVICE, [n_points][k][ts->n_tasks] or NULL; out_sched DEVICE, [n_points][k]
+ *              [n_tasksets]; k = number of requested analyses, in the order of the constants below
+ *   everything else as for gcaps_rta_batch.
+ */
+#define GCAPS_ANALYSIS_GCAPS_SUSPEND 1
+#define GCAPS_ANALYSIS_GCAPS_BUSY 2
+#define GCAPS_ANALYSIS_RR_SUSPEND 4
+#define GCAPS_ANALYSIS_RR_BUSY 8
+int gcaps_rta_multi_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int analyses, int flags,
+                          int n_points, const int64_t *timeslice_us,
+                          const int64_t *ctx_switch_overhead_us, int64_t *out_wcrt,
+                          uint8_t *out_sched, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * gcaps_rta_batch_static -- gcaps_rta_batch for callers that are not able to allocate device
  * memory.  (The paper has no counterpart: this is a convenience of this library, not a step of
  * the analysis.)

@@ -118,6 +118,21 @@ def analyse_sweep(batch, policy: int, timeslices_us, overheads_us, iter_cap: int
     return wcrt, sched
 
 
+def analyse_multi(batch, policies, timeslices_us, overheads_us, iter_cap: int = ITER_CAP):
+    """Several analyses (``policies``: policy | flags words) of the same batch under several
+    ``(timeslice, overhead)`` pairs: by definition one independent ``analyse`` per combination.
+    Returns ``(wcrt, sched)`` of shapes ``[n_params, n_policies, n_tasks]`` and
+    ``[n_params, n_policies, n_tasksets]``."""
+    n_tasksets = np.asarray(batch.task_off).shape[0] - 1
+    n_tasks = np.asarray(batch.period).shape[0]
+    wcrt = np.full((len(overheads_us), len(policies), n_tasks), WCRT_INVALID, np.int64)
+    sched = np.full((len(overheads_us), len(policies), n_tasksets), SCHED_INVALID, np.uint8)
+    for q, (L, ovh) in enumerate(zip(timeslices_us, overheads_us)):
+        for j, pol in enumerate(policies):
+            analyse(batch, pol, int(L), int(ovh), iter_cap=iter_cap, out=(wcrt[q, j], sched[q, j]))
+    return wcrt, sched
+
+
 def validate(batch) -> np.ndarray:
     """Per-taskset domain check; 0 = valid, else a bit mask (1 task range, 2 segment range,
     4 period, 8 deadline, 16 core, 32 WCET)."""

@@ -30,11 +30,15 @@ MAX_TIME = 1 << 40
 OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NO_DEVICE, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5
 STATIC_MAX_TASKSETS = 65536
 MAX_SWEEP = 32
+# analyses of rta_multi, in result order
+GCAPS_SUSPEND, GCAPS_BUSY, RR_SUSPEND, RR_BUSY = 1, 2, 4, 8
+ANALYSIS_POLICY = {GCAPS_SUSPEND: POLICY_GCAPS, GCAPS_BUSY: POLICY_GCAPS | BUSY,
+                   RR_SUSPEND: POLICY_RR, RR_BUSY: POLICY_RR | BUSY}
 
 EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host",
            "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
            "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static",
-           "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch", "gcaps_rta_sweep_batch",
+           "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch", "gcaps_rta_sweep_batch", "gcaps_rta_multi_batch",
            "gcaps_gen_workspace_bytes", "gcaps_gen_count", "gcaps_gen_fill")
 
 _p64 = ctypes.POINTER(ctypes.c_int64)
@@ -93,6 +97,10 @@ def load_library(path: Optional[str] = None):
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int, _p64, _p64,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         lib.gcaps_rta_sweep_batch.restype = ctypes.c_int
+        lib.gcaps_rta_multi_batch.argtypes = [
+            ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int, _p64, _p64,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        lib.gcaps_rta_multi_batch.restype = ctypes.c_int
         lib.gcaps_gen_workspace_bytes.argtypes = [ctypes.c_int64]
         lib.gcaps_gen_workspace_bytes.restype = ctypes.c_size_t
         lib.gcaps_gen_count.argtypes = [ctypes.POINTER(IntParams), ctypes.c_int64, ctypes.c_int64,
@@ -194,6 +202,35 @@ def rta_sweep(ts: DeviceTasksets, policy: int, timeslices_us, overheads_us, want
             workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
         st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_sweep_batch(ctypes.byref(ts.c), ts.n_tasksets, policy, k, Ls, ov,
+                                       out_wcrt.data_ptr() if out_wcrt is not None else None,
+                                       out_sched.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                       st.cuda_stream)
+    _check(rc)
+    return out_wcrt, out_sched
+
+
+def rta_multi(ts: DeviceTasksets, analyses: int, timeslices_us=(1024,), overheads_us=(0,), flags: int = 0,
+              want_wcrt: bool = True, out_wcrt=None, out_sched=None, workspace=None, stream=None):
+    """gcaps_rta_multi_batch: the analyses named in ``analyses`` (OR of ``GCAPS_SUSPEND``,
+    ``GCAPS_BUSY``, ``RR_SUSPEND``, ``RR_BUSY``) for every ``(timeslice, overhead)`` pair, one pass
+    over the resident batch.  Returns ``(out_wcrt, out_sched)`` CUDA tensors of shapes
+    ``[n_points, k, n_tasks]`` (None with ``want_wcrt=False``) and ``[n_points, k, n_tasksets]``,
+    ``k`` analyses in the order of the four constants."""
+    import torch
+    lib = load_library()
+    dev = ts.t["task_off"].device
+    n_pts, k = len(overheads_us), bin(analyses & 15).count("1")
+    Ls = (ctypes.c_int64 * n_pts)(*[int(x) for x in timeslices_us]) if timeslices_us is not None else None
+    ov = (ctypes.c_int64 * n_pts)(*[int(x) for x in overheads_us])
+    with torch.cuda.device(dev):
+        if out_wcrt is None and want_wcrt:
+            out_wcrt = torch.empty((n_pts, k, ts.n_tasks), dtype=torch.int64, device=dev)
+        if out_sched is None:
+            out_sched = torch.empty((n_pts, k, max(ts.n_tasksets, 0)), dtype=torch.uint8, device=dev)
+        if workspace is None:
+            workspace = torch.empty(max(workspace_bytes(ts.n_tasksets), 256), dtype=torch.uint8, device=dev)
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        rc = lib.gcaps_rta_multi_batch(ctypes.byref(ts.c), ts.n_tasksets, analyses, flags, n_pts, Ls, ov,
                                        out_wcrt.data_ptr() if out_wcrt is not None else None,
                                        out_sched.data_ptr(), workspace.data_ptr(), workspace.numel(),
                                        st.cuda_stream)

@@ -430,6 +430,12 @@ __device__ __forceinline__ void prefix_step(const i64 *__restrict__ X0, const i6
   }
 }
 
+// An analysis mode known at compile time (converts to int like a run-time mode does).
+template <int V>
+struct ModeTag {
+  __host__ __device__ constexpr operator int() const { return V; }
+};
+
 // MODE: 0 GCAPS self-suspension, 1 GCAPS busy-waiting, 2 RR self-suspension, 3 RR busy-waiting.
 // Returns false, having written nothing, if the taskset is not eligible for 32-bit arithmetic
 // (or is invalid): the caller then runs the exact 64-bit path, which also does the validation.
@@ -443,7 +449,12 @@ __device__ __forceinline__ void prefix_step(const i64 *__restrict__ X0, const i6
 // SWEEP: the taskset is staged, ordered and aggregated once and then analysed under every
 // (timeslice, overhead) pair of `sw`; pair q writes out_wcrt + q * n_tasks (skipped when out_wcrt
 // is null) and out_sched + q * n_tasksets.
-template <int LPT, int SLOTS, int MODE, bool SWEEP = false>
+//
+// MASK: bit m set = analysis MODE m is run.  One bit: the plain kernels.  Several bits (always
+// with SWEEP): every (timeslice, overhead) pair is analysed under each mode of MASK that
+// sw->enabled also names, in ascending mode order; the k-th analysis of a taskset writes result
+// block k (out_wcrt + k * n_tasks, out_sched + k * n_tasksets).
+template <int LPT, int SLOTS, int MASK, bool SWEEP = false>
 __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane,
                                              unsigned int gmask, const SweepArgs *sw = nullptr) {
   typedef FastLayout<LPT, SLOTS> Lay;
@@ -451,7 +462,9 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   constexpr int MAXN = Lay::MAXN, CAP = Lay::CAP;
   constexpr int BC = SLOTS <= 2 ? SLOTS : 2;  // prefix blocks whose loads are issued together
   constexpr int BG = 1;
-  constexpr bool kGcaps = MODE < 2;
+  constexpr bool kAnyGcaps = (MASK & 3) != 0;
+  constexpr bool kMulti = (MASK & (MASK - 1)) != 0;
+  static_assert(!kMulti || SWEEP, "several analyses per taskset use the sweep loop");
   const bool literal = (p.policy & GCAPS_RTA_LITERAL) != 0;
   const bool best_effort = (p.policy & GCAPS_RTA_BEST_EFFORT) != 0;
   uint4 *info = reinterpret_cast<uint4 *>(buf + Lay::kInfo);
@@ -613,29 +626,18 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   int n_gpu = 0;  // N_g
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(gmask, eta[s] > 0));
-  if (kGcaps) {  // 2 * eps * eta must stay below 2^26 (eta < 64, eps < 2^20: no overflow here)
+  if (kAnyGcaps) {  // 2 * eps * eta must stay below 2^26 (eta < 64, eps < 2^20: no overflow here)
     const u32 ovh_max = SWEEP ? (u32)sw->max_ovh : (u32)p.ovh;
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) bad |= (2 * ovh_max * eta[s]) >> 26;
   }
   if (__any_sync(gmask, bad != 0)) return false;
-  u32 magic[SLOTS], shift[SLOTS];  // reciprocal of T_h by rank, made when the slot is first needed
-#pragma unroll
-  for (int s = 0; s < SLOTS; ++s) magic[s] = 0, shift[s] = 0;
-  int slots_made = 0;
-  u32 sl[SLOTS];  // RR: slices of the task's pure GPU parts (Eq. 3), by position
-#pragma unroll
-  for (int s = 0; s < SLOTS; ++s) sl[s] = 0;
-  u32 *Ps = SWEEP ? Q1 : Q0;  // running sums of the slice counts (a sweep keeps Q0 for the exchange)
-  const int n_points = SWEEP ? sw->n : 1;
-  for (int q = 0; q < n_points; ++q) {
-  const i64 L64 = SWEEP ? sw->q[q].L : p.L;
-  const u32 ovh = SWEEP ? (u32)sw->q[q].ovh : (u32)p.ovh;  // the fast path needs eps, theta < 2^20
-  const u32 l_mode = SWEEP ? sw->q[q].l_mode : p.l_mode, l_magic = SWEEP ? sw->q[q].l_magic : p.l_magic;
-  const u32 l_shift = SWEEP ? sw->q[q].l_shift : p.l_shift;
-  i64 *const out_wcrt = SWEEP ? (p.out_wcrt ? p.out_wcrt + (i64)q * p.n_tasks : nullptr) : p.out_wcrt;
-  uint8_t *const out_sched = SWEEP ? p.out_sched + (i64)q * p.n_tasksets : p.out_sched;
-  if (!kGcaps && (!SWEEP || q == 0 || sw->q[q].L != sw->q[q - 1].L)) {
+  const int n_rt_all = (int)Q0[-2];  // real-time tasks: the ranks that are analysed
+  uint4 *xch = reinterpret_cast<uint4 *>(Q0);  // by rank: T, C+G^m, G^e, S  (Q0 is dead by now)
+
+  // Eq. 3: running sums of the slices of every pure GPU part for timeslice L (values already
+  // checked) into Ps
+  auto slice_sums = [&](u32 *Ps, i64 L64, u32 l_mode, u32 l_magic, u32 l_shift) {
     // Eq. 3: slices of every pure GPU part, summed per task (values already checked)
     const bool inside = slice_is_inside(gfirst, Ng, pare, p.n_gsegs);
     u32 carry = 0;
@@ -681,59 +683,37 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       }
     }
     __syncwarp(gmask);
-#pragma unroll
-    for (int s = 0; s < SLOTS; ++s) sl[s] = Ps[g1[s] - 1 + pare] - Ps[g0[s] - 1 + pare];
-    __syncwarp(gmask);
-  }
-  // ---- constants of Eq. 1 that do not depend on R ------------------------------------------
-  u32 base[SLOTS];
-#pragma unroll
-  for (int s = 0; s < SLOTS; ++s) {
-    if (kGcaps) {
-      S[s] = 2 * ovh * eta[s];                                 // eta < 64: below 2^27
-      base[s] = A[s] + Ge[s] + S[s] + (eta[s] + 1) * ovh;        // C_i + G*_i + B^C_i, below 2^29
-    } else {
-      const u64 slices = sl[s];
-      const u64 lt = (u64)L64 + ovh;  // <= 2^41
-      u64 B = slices == 0 ? 0 : (lt >= kFastClamp ? kFastClamp : lt * slices);  // < 2^26 * 2^32
-      if (B > kFastClamp) B = kFastClamp;
-      S[s] = (u32)B;
-      const u64 b64 = (u64)A[s] + Ge[s] + (eta[s] > 0 ? B * (u64)(n_gpu - 1) : 0);  // Lemma 1
-      base[s] = b64 > (u64)(2 * kFastClamp) ? 2 * kFastClamp : (u32)b64;
-    }
-    base[s] = base[s] > 2 * kFastClamp ? 2 * kFastClamp : base[s];
-  }
-  __syncwarp(gmask);
-  // ---- move every task to the lane that owns its rank -------------------------------------
-  uint4 *xch = reinterpret_cast<uint4 *>(Q0);  // by rank: T, C+G^m, G^e, S  (Q0 is dead by now)
-#pragma unroll
-  for (int s = 0; s < SLOTS; ++s) {
-    if (lane + LPT * s < n) {
-      *(reinterpret_cast<uint2 *>(&info[rank[s]]) + 1) =
-          make_uint2(base[s], (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u));
-      xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], S[s]);
-    }
-  }
-  __syncwarp(gmask);
-  // by rank from here on: period - 1, C+G^m, G^e, S, the two weights of the analysis' pairs
-  u32 Tm1[SLOTS], Ar[SLOTS], Ger[SLOTS], Wa[SLOTS], Wb[SLOTS], pos_of[SLOTS], core[SLOTS];
+  };
+
+  // The recurrence of Eq. 1 for every real-time task in rank order under analysis MODE, once the
+  // tasks sit in the lanes of their ranks: Sr = 2*eps*eta (GCAPS) or (L+theta)*slices (RR) of this
+  // lane's tasks, info[rank].z = base.  Writes out_wcrt (unless null in a sweep) and out_sched.
+  auto recurrence = [&](auto mode_tag, i64 *out_wcrt, uint8_t *out_sched) {
+  constexpr int MODE = mode_tag;  // a ModeTag: every analysis of a kernel gets its own copy
+  const int n_rt = n_rt_all;
+  // by rank from here on: period - 1, C+G^m, G^e, core, position, GPU-using, and the two weights
+  // of the analysis' pairs
+  u32 Tm1[SLOTS], Ar[SLOTS], Ger[SLOTS], pos_of[SLOTS], core[SLOTS], Wa[SLOTS], Wb[SLOTS];
   bool gpu[SLOTS];
+  u32 magic[SLOTS], shift[SLOTS];  // reciprocal of T_h, made when the slot is first needed
+  int slots_made = 0;
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     const int r = lane + LPT * s;
     const uint4 x = r < n ? xch[r] : make_uint4(2u, 0u, 0u, 0u);
     const uint4 f = r < n ? info[r] : make_uint4(0u, 0xffffffffu, 0u, 0u);
-    const u32 Sr = x.w;
+    const u32 Sr = x.w;  // 2*eps*eta (GCAPS) or (L+theta)*slices (RR) of this rank's task
     Tm1[s] = x.x - 1, Ar[s] = x.y, Ger[s] = x.z;
     core[s] = f.y, pos_of[s] = f.w & 0xffffu, gpu[s] = (f.w & 0x10000u) != 0;
+    magic[s] = 0, shift[s] = 0;
     if (MODE == 0) {
       Wa[s] = Ar[s] + (gpu[s] ? Sr : 0u);    // Lemma 15: C_h, or C_h + G^{m*}_h
       Wb[s] = gpu[s] ? Ger[s] + Sr : 0u;     // Lemma 13, other cores: G^{e*}_h
     } else if (MODE == 1) {
-      Wa[s] = Ar[s];                         // Lemma 12
+      Wa[s] = Ar[s];                            // Lemma 12
       Wb[s] = gpu[s] ? Ger[s] + Sr : 0u;     // Lemmas 10, 11: G^{e*}_h
     } else {
-      Wa[s] = Ar[s];                         // Lemmas 5, 7
+      Wa[s] = Ar[s];                            // Lemmas 5, 7
       Wb[s] = gpu[s] ? Sr : 0u;              // Lemma 4: (L+theta) * slices
     }
   }
@@ -742,7 +722,6 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   u32 Jc[SLOTS], Jg[SLOTS];               // jitters with T_h - 1 folded in (ceiling)
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) Jc[s] = Jg[s] = Tm1[s];
-  const int n_rt = (int)Q0[-2];  // real-time tasks: the ranks that are analysed
   int n_done = n_rt;
   int verdict = 0;
   for (int pos = 0; pos < n_rt; ++pos) {
@@ -848,7 +827,127 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   }
   if (lane == 0) out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
   __syncwarp(gmask);
-  }  // next (timeslice, overhead) pair
+  };  // recurrence
+
+  if constexpr (!SWEEP) {
+    // ---- one analysis: constants by position, then everything moves to the rank's lane ---------
+    constexpr int MODE = (MASK & 1) ? 0 : (MASK & 2) ? 1 : (MASK & 4) ? 2 : 3;
+    constexpr bool kGcaps = MODE < 2;
+    const u32 ovh = (u32)p.ovh;  // the fast path needs eps, theta < 2^20
+    u32 sl[SLOTS];               // RR: slices of the task's pure GPU parts (Eq. 3)
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) sl[s] = 0;
+    if (!kGcaps) {
+      slice_sums(Q0, p.L, p.l_mode, p.l_magic, p.l_shift);
+      __syncwarp(gmask);
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s) sl[s] = Q0[g1[s] - 1 + pare] - Q0[g0[s] - 1 + pare];
+      __syncwarp(gmask);
+    }
+    u32 base[SLOTS];
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      if (kGcaps) {
+        S[s] = 2 * ovh * eta[s];                                 // eta < 64: below 2^27
+        base[s] = A[s] + Ge[s] + S[s] + (eta[s] + 1) * ovh;        // C_i + G*_i + B^C_i, below 2^29
+      } else {
+        const u64 slices = sl[s];
+        const u64 lt = (u64)p.L + ovh;  // <= 2^41
+        u64 B = slices == 0 ? 0 : (lt >= kFastClamp ? kFastClamp : lt * slices);  // < 2^26 * 2^32
+        if (B > kFastClamp) B = kFastClamp;
+        S[s] = (u32)B;
+        const u64 b64 = (u64)A[s] + Ge[s] + (eta[s] > 0 ? B * (u64)(n_gpu - 1) : 0);  // Lemma 1
+        base[s] = b64 > (u64)(2 * kFastClamp) ? 2 * kFastClamp : (u32)b64;
+      }
+      base[s] = base[s] > 2 * kFastClamp ? 2 * kFastClamp : base[s];
+    }
+    __syncwarp(gmask);
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      if (lane + LPT * s < n) {
+        *(reinterpret_cast<uint2 *>(&info[rank[s]]) + 1) =
+            make_uint2(base[s], (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u));
+        xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], S[s]);
+      }
+    }
+    __syncwarp(gmask);
+    recurrence(ModeTag<MODE>(), p.out_wcrt, p.out_sched);
+  } else {
+    // ---- several analyses: the tasks move to the rows of their ranks once; for every analysis
+    // the lane of a rank then makes that task's S and base from the row and the recurrence
+    // starts from the rows again, so nothing per task is held in registers across analyses ------
+    // second row by rank: GPU segment range (11 bits each) and number of GPU segments (6 bits)
+    // packed in .x, slices of Eq. 3 for the timeslice sl_L in .y
+    uint2 *xch2 = reinterpret_cast<uint2 *>(Q0 + 4 * MAXN);
+    static_assert(Lay::CAP <= 2048 && Lay::CAP >= 6 * MAXN, "packed segment range, room for the second row");
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      if (lane + LPT * s < n) {
+        info[rank[s]].w = (u32)(lane + LPT * s) | (eta[s] > 0 ? 0x10000u : 0u);
+        xch[rank[s]] = make_uint4(T[s], A[s], Ge[s], 0u);
+        xch2[rank[s]] = make_uint2((u32)g0[s] | ((u32)g1[s] << 11) | (eta[s] << 22), 0u);
+      }
+    }
+    __syncwarp(gmask);
+    i64 sl_L = -1;
+    constexpr bool kMultiModes = (MASK & (MASK - 1)) != 0;
+    const int enabled = kMultiModes ? sw->enabled : MASK;
+    for (int q = 0; q < sw->n; ++q) {
+      const i64 L64 = sw->q[q].L;
+      const u32 ovh = (u32)sw->q[q].ovh;  // the fast path needs eps, theta < 2^20
+      auto analyse_as = [&](auto mode_tag) {
+        constexpr int MODE = mode_tag;
+        constexpr bool kGcaps = MODE < 2;
+        const int block = q * sw->block_stride + sw->block_of_mode[MODE];
+        i64 *const out_wcrt = p.out_wcrt ? p.out_wcrt + (i64)block * p.n_tasks : nullptr;
+        uint8_t *const out_sched = p.out_sched + (i64)block * p.n_tasksets;
+        if (!kGcaps && L64 != sl_L) {
+          sl_L = L64;
+          slice_sums(Q1, L64, sw->q[q].l_mode, sw->q[q].l_magic, sw->q[q].l_shift);
+          __syncwarp(gmask);
+#pragma unroll
+          for (int s = 0; s < SLOTS; ++s) {
+            const int r = lane + LPT * s;
+            if (r < n) {
+              const u32 g = xch2[r].x;
+              xch2[r].y = Q1[(int)((g >> 11) & 0x7ffu) - 1 + pare] - Q1[(int)(g & 0x7ffu) - 1 + pare];
+            }
+          }
+        }
+#pragma unroll
+        for (int s = 0; s < SLOTS; ++s) {
+          const int r = lane + LPT * s;
+          if (r < n) {
+            const uint4 x = xch[r];
+            const uint2 g = xch2[r];
+            const u32 eta_r = g.x >> 22;
+            u32 Sr, base;
+            if (kGcaps) {
+              Sr = 2 * ovh * eta_r;                                 // eta < 64: below 2^27
+              base = x.y + x.z + Sr + (eta_r + 1) * ovh;             // C_i + G*_i + B^C_i, below 2^29
+            } else {
+              const u64 slices = g.y;
+              const u64 lt = (u64)L64 + ovh;  // <= 2^41
+              u64 B = slices == 0 ? 0 : (lt >= kFastClamp ? kFastClamp : lt * slices);
+              if (B > kFastClamp) B = kFastClamp;
+              Sr = (u32)B;
+              const u64 b64 = (u64)x.y + x.z + (eta_r > 0 ? B * (u64)(n_gpu - 1) : 0);  // Lemma 1
+              base = b64 > (u64)(2 * kFastClamp) ? 2 * kFastClamp : (u32)b64;
+            }
+            base = base > 2 * kFastClamp ? 2 * kFastClamp : base;
+            xch[r].w = Sr;
+            info[r].z = base;
+          }
+        }
+        __syncwarp(gmask);
+        recurrence(mode_tag, out_wcrt, out_sched);
+      };
+      if ((MASK & 1) && (enabled & 1)) analyse_as(ModeTag<0>());
+      if ((MASK & 2) && (enabled & 2)) analyse_as(ModeTag<1>());
+      if ((MASK & 4) && (enabled & 4)) analyse_as(ModeTag<2>());
+      if ((MASK & 8) && (enabled & 8)) analyse_as(ModeTag<3>());
+    }
+  }
   return true;
 }
 
@@ -878,7 +977,7 @@ __host__ __device__ constexpr int min_blocks(int slots) {
 // LPT lanes; every group analyses one taskset at a time.  Warps pull chunks of taskset indices
 // from the bin's counter; the index, task range and first segment offsets of the next chunk are
 // fetched while the current one is analysed.
-template <int LPT, int SLOTS, int MODE, bool SWEEP = false>
+template <int LPT, int SLOTS, int MASK, bool SWEEP = false>
 __device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf, Ahead *ahead,
                                         const SweepArgs *sw = nullptr) {
   typedef FastLayout<LPT, SLOTS> Lay;
@@ -956,20 +1055,28 @@ __device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf
           prefetch_l2(p.gseg_misc + me.g_lo + e), prefetch_l2(p.gseg_exec + me.g_lo + e);
         bool done = false;
         if (fast_call && (me.packed >> 31) != 0)
-          done = analyse_fast<LPT, SLOTS, MODE, SWEEP>(p, t, me.a, n, buf, lane, gmask, sw);
+          done = analyse_fast<LPT, SLOTS, MASK, SWEEP>(p, t, me.a, n, buf, lane, gmask, sw);
         __syncwarp(gmask);
         if (!done && !SWEEP) {
           // the exact path reads task_off again and validates everything itself
           analyse_taskset<LPT, MAXN>(p, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, gmask);
         }
         if (!done && SWEEP) {  // the exact path once per (timeslice, overhead) pair
+          constexpr bool kMulti = (MASK & (MASK - 1)) != 0;
+          const int enabled = kMulti ? sw->enabled : MASK;
           for (int q = 0; q < sw->n; ++q) {
-            KParams pq = p;
-            pq.L = sw->q[q].L, pq.ovh = sw->q[q].ovh;
-            pq.out_wcrt = p.out_wcrt ? p.out_wcrt + (i64)q * p.n_tasks : nullptr;
-            pq.out_sched = p.out_sched + (i64)q * p.n_tasksets;
-            analyse_taskset<LPT, MAXN>(pq, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, gmask);
-            __syncwarp(gmask);
+            for (int m = 0; m < 4; ++m) {
+              if (!((MASK & enabled) >> m & 1)) continue;
+              const int block = q * sw->block_stride + sw->block_of_mode[m];
+              KParams pq = p;
+              pq.policy = (p.policy & ~(0xff | GCAPS_RTA_BUSY)) | (m >= 2 ? GCAPS_POLICY_RR : GCAPS_POLICY_GCAPS) |
+                          ((m & 1) ? GCAPS_RTA_BUSY : 0);
+              pq.L = sw->q[q].L, pq.ovh = sw->q[q].ovh;
+              pq.out_wcrt = p.out_wcrt ? p.out_wcrt + (i64)block * p.n_tasks : nullptr;
+              pq.out_sched = p.out_sched + (i64)block * p.n_tasksets;
+              analyse_taskset<LPT, MAXN>(pq, t, *reinterpret_cast<GroupSmem<MAXN> *>(buf), lane, gmask);
+              __syncwarp(gmask);
+            }
           }
         }
       }
@@ -998,10 +1105,10 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(3)) rta_small_kernel
   extern __shared__ __align__(16) unsigned char smem_raw[];
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
-  run_bin<16, 2, MODE>(p, 3, warp_buf, ahead);
-  run_bin<8, 3, MODE>(p, 2, warp_buf, ahead);
-  run_bin<8, 2, MODE>(p, 1, warp_buf, ahead);
-  run_bin<8, 1, MODE>(p, 0, warp_buf, ahead);
+  run_bin<16, 2, 1 << MODE>(p, 3, warp_buf, ahead);
+  run_bin<8, 3, 1 << MODE>(p, 2, warp_buf, ahead);
+  run_bin<8, 2, 1 << MODE>(p, 1, warp_buf, ahead);
+  run_bin<8, 1, 1 << MODE>(p, 0, warp_buf, ahead);
 }
 
 // One bin of larger tasksets (a warp per taskset, 2, 3, 4, 6 or 8 tasks per lane) per launch.
@@ -1011,31 +1118,31 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kern
   constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
-  run_bin<32, SLOTS, MODE>(p, bin, warp_buf, ahead);
+  run_bin<32, SLOTS, 1 << MODE>(p, bin, warp_buf, ahead);
 }
 
 // The same launches for a fused sweep: every taskset is read once and analysed under all the
 // (timeslice, overhead) pairs of `sw`.
-template <int MODE>
-__global__ void __launch_bounds__(kBlockThreads, 4)
+template <int MASK>
+__global__ void __launch_bounds__(kBlockThreads, min_blocks(3))
 rta_small_sweep_kernel(KParams p, const __grid_constant__ SweepArgs sw) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
-  run_bin<16, 2, MODE, true>(p, 3, warp_buf, ahead, &sw);
-  run_bin<8, 3, MODE, true>(p, 2, warp_buf, ahead, &sw);
-  run_bin<8, 2, MODE, true>(p, 1, warp_buf, ahead, &sw);
-  run_bin<8, 1, MODE, true>(p, 0, warp_buf, ahead, &sw);
+  run_bin<16, 2, MASK, true>(p, 3, warp_buf, ahead, &sw);
+  run_bin<8, 3, MASK, true>(p, 2, warp_buf, ahead, &sw);
+  run_bin<8, 2, MASK, true>(p, 1, warp_buf, ahead, &sw);
+  run_bin<8, 1, MASK, true>(p, 0, warp_buf, ahead, &sw);
 }
 
-template <int SLOTS, int MODE>
-__global__ void __launch_bounds__(kBlockThreads, (SLOTS <= 4 ? 4 : min_blocks(SLOTS)))
+template <int SLOTS, int MASK>
+__global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS))
 rta_big_sweep_kernel(KParams p, int bin, const __grid_constant__ SweepArgs sw) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
-  run_bin<32, SLOTS, MODE, true>(p, bin, warp_buf, ahead, &sw);
+  run_bin<32, SLOTS, MASK, true>(p, bin, warp_buf, ahead, &sw);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1205,45 +1312,70 @@ cudaError_t launch_all_bins(const KParams &p, int sm_count, cudaStream_t st) {
   return e;
 }
 
-template <int SLOTS, int MODE>
+template <int SLOTS, int MASK>
 cudaError_t launch_big_sweep(const KParams &p, const SweepArgs &sw, int bin, int sm_count, cudaStream_t st) {
   constexpr int kWarps = kBlockThreads / 32;
   static int blocks_per_sm[64] = {0};
   const size_t smem = sizeof(u32) * (bin_warp_words<32, SLOTS>() + kAheadWords) * kWarps;
-  return launch_persistent(rta_big_sweep_kernel<SLOTS, MODE>, blocks_per_sm, smem,
+  return launch_persistent(rta_big_sweep_kernel<SLOTS, MASK>, blocks_per_sm, smem,
                            (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p, bin, sw);
 }
 
-template <int MODE>
+template <int MASK>
 cudaError_t launch_all_bins_sweep(const KParams &p, const SweepArgs &sw, int sm_count, cudaStream_t st) {
   constexpr int kWarps = kBlockThreads / 32;
   static int blocks_per_sm[64] = {0};
   const size_t smem = sizeof(u32) * kSmallWarpWords * kWarps;
-  cudaError_t e = launch_persistent(rta_small_sweep_kernel<MODE>, blocks_per_sm, smem,
+  cudaError_t e = launch_persistent(rta_small_sweep_kernel<MASK>, blocks_per_sm, smem,
                                     (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p, sw);
-  if (e == cudaSuccess) e = launch_big_sweep<2, MODE>(p, sw, 4, sm_count, st);
-  if (e == cudaSuccess) e = launch_big_sweep<3, MODE>(p, sw, 5, sm_count, st);
-  if (e == cudaSuccess) e = launch_big_sweep<4, MODE>(p, sw, 6, sm_count, st);
-  if (e == cudaSuccess) e = launch_big_sweep<6, MODE>(p, sw, 7, sm_count, st);
-  if (e == cudaSuccess) e = launch_big_sweep<8, MODE>(p, sw, 8, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<2, MASK>(p, sw, 4, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<3, MASK>(p, sw, 5, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<4, MASK>(p, sw, 6, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<6, MASK>(p, sw, 7, sm_count, st);
+  if (e == cudaSuccess) e = launch_big_sweep<8, MASK>(p, sw, 8, sm_count, st);
   return e;
 }
 
-// Plan + analysis launches of one call; `sw` non-null: the fused sweep.
+cudaError_t launch_sweep_set(const KParams &p, const SweepArgs &sw, int sm_count, cudaStream_t st) {
+  switch (sw.enabled) {
+    case 1: return launch_all_bins_sweep<1>(p, sw, sm_count, st);
+    case 2: return launch_all_bins_sweep<2>(p, sw, sm_count, st);
+    case 4: return launch_all_bins_sweep<4>(p, sw, sm_count, st);
+    case 8: return launch_all_bins_sweep<8>(p, sw, sm_count, st);
+    case 5: return launch_all_bins_sweep<5>(p, sw, sm_count, st);   // GCAPS + RR, self-suspension
+    case 10: return launch_all_bins_sweep<10>(p, sw, sm_count, st);  // GCAPS + RR, busy-waiting
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+// Plan + analysis launches of one call.  `sw` null: one analysis (p.policy).  Otherwise the
+// analyses named in `analyses` (bit m = mode m) for every pair of `sw`: the self-suspension
+// modes in one set of launches, the busy-waiting modes in another (the plan is shared, the work
+// counters are cleared in between).
 int enqueue_batch(KParams p, void *workspace, size_t workspace_bytes, int sm_count, cudaStream_t st,
-                  const SweepArgs *sw = nullptr) {
+                  const SweepArgs *sw = nullptr, int analyses = 0) {
   if (p.n_tasksets == 0) return GCAPS_OK;
   const int rc = enqueue_plan(p, workspace, workspace_bytes, st);
   if (rc != GCAPS_OK) return rc;
   cudaError_t e = cudaGetLastError();
-  if (e == cudaSuccess) {
+  if (e == cudaSuccess && sw) {
+    SweepArgs set = *sw;
+    set.block_stride = __builtin_popcount(analyses);
+    for (int m = 0, k = 0; m < 4; ++m) {
+      set.block_of_mode[m] = k;
+      k += (analyses >> m) & 1;
+    }
+    bool first = true;
+    for (int half = 0; half < 2 && e == cudaSuccess; ++half) {
+      set.enabled = analyses & (half == 0 ? 5 : 10);
+      if (set.enabled == 0) continue;
+      if (!first) e = cudaMemsetAsync(p.hdr->next, 0, sizeof(p.hdr->next), st);
+      first = false;
+      if (e == cudaSuccess) e = launch_sweep_set(p, set, sm_count, st);
+    }
+  } else if (e == cudaSuccess) {
     const bool rr = (p.policy & 0xff) == GCAPS_POLICY_RR, busy = (p.policy & GCAPS_RTA_BUSY) != 0;
-    if (sw) {
-      if (!rr && !busy) e = launch_all_bins_sweep<0>(p, *sw, sm_count, st);
-      else if (!rr) e = launch_all_bins_sweep<1>(p, *sw, sm_count, st);
-      else if (!busy) e = launch_all_bins_sweep<2>(p, *sw, sm_count, st);
-      else e = launch_all_bins_sweep<3>(p, *sw, sm_count, st);
-    } else if (!rr && !busy) e = launch_all_bins<0>(p, sm_count, st);
+    if (!rr && !busy) e = launch_all_bins<0>(p, sm_count, st);
     else if (!rr) e = launch_all_bins<1>(p, sm_count, st);
     else if (!busy) e = launch_all_bins<2>(p, sm_count, st);
     else e = launch_all_bins<3>(p, sm_count, st);
@@ -1297,14 +1429,17 @@ int gcaps_rta_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
   return enqueue_batch(p, workspace, workspace_bytes, di.sm_count, (cudaStream_t)stream);
 }
 
-int gcaps_rta_sweep_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy, int n_points,
-                          const int64_t *timeslice_us, const int64_t *ctx_switch_overhead_us,
-                          int64_t *out_wcrt, uint8_t *out_sched, void *workspace,
-                          size_t workspace_bytes, void *stream) {
+int gcaps_rta_multi_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int analyses, int flags,
+                          int n_points, const int64_t *timeslice_us,
+                          const int64_t *ctx_switch_overhead_us, int64_t *out_wcrt,
+                          uint8_t *out_sched, void *workspace, size_t workspace_bytes, void *stream) {
+  if (analyses < 1 || analyses > 15 || (flags & ~(GCAPS_RTA_LITERAL | GCAPS_RTA_BEST_EFFORT)))
+    return GCAPS_ERR_INVALID_ARG;
   if (n_points < 1 || n_points > GCAPS_RTA_MAX_SWEEP || !ctx_switch_overhead_us)
     return GCAPS_ERR_INVALID_ARG;
-  const bool rr = (policy & 0xff) == GCAPS_POLICY_RR;
+  const bool rr = (analyses & (GCAPS_ANALYSIS_RR_SUSPEND | GCAPS_ANALYSIS_RR_BUSY)) != 0;
   if (rr && !timeslice_us) return GCAPS_ERR_INVALID_ARG;
+  const int policy = (rr ? GCAPS_POLICY_RR : GCAPS_POLICY_GCAPS) | flags;  // (for the argument checks)
   SweepArgs sw;
   memset(&sw, 0, sizeof(sw));
   sw.n = n_points;
@@ -1325,7 +1460,20 @@ int gcaps_rta_sweep_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int po
   if (rc != GCAPS_OK) return rc;
   KParams p;
   fill_params(&p, ts, n_tasksets, policy, sw.q[0].L, sw.q[0].ovh, out_wcrt, out_sched);
-  return enqueue_batch(p, workspace, workspace_bytes, di.sm_count, (cudaStream_t)stream, &sw);
+  return enqueue_batch(p, workspace, workspace_bytes, di.sm_count, (cudaStream_t)stream, &sw, analyses);
+}
+
+int gcaps_rta_sweep_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy, int n_points,
+                          const int64_t *timeslice_us, const int64_t *ctx_switch_overhead_us,
+                          int64_t *out_wcrt, uint8_t *out_sched, void *workspace,
+                          size_t workspace_bytes, void *stream) {
+  const int pol = policy & 0xff;
+  if (pol != GCAPS_POLICY_GCAPS && pol != GCAPS_POLICY_RR) return GCAPS_ERR_INVALID_ARG;
+  if (policy & ~(0xff | GCAPS_RTA_BUSY | GCAPS_RTA_LITERAL | GCAPS_RTA_BEST_EFFORT)) return GCAPS_ERR_INVALID_ARG;
+  const int mode = (pol == GCAPS_POLICY_RR ? 2 : 0) + ((policy & GCAPS_RTA_BUSY) ? 1 : 0);
+  return gcaps_rta_multi_batch(ts, n_tasksets, 1 << mode, policy & (GCAPS_RTA_LITERAL | GCAPS_RTA_BEST_EFFORT),
+                               n_points, timeslice_us, ctx_switch_overhead_us, out_wcrt, out_sched,
+                               workspace, workspace_bytes, stream);
 }
 
 int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,

@@ -57,6 +57,11 @@ struct SweepPoint {
 };
 struct SweepArgs {
   int n;        // pairs, 1 .. GCAPS_RTA_MAX_SWEEP
+  int enabled;  // analyses this launch runs per pair: bit m = mode m (0 GCAPS self-suspension,
+                // 1 GCAPS busy-waiting, 2 RR self-suspension, 3 RR busy-waiting)
+  // the analysis of pair q under mode m writes result block q * block_stride + block_of_mode[m]
+  int block_stride;
+  int block_of_mode[4];
   i64 max_ovh;  // largest overhead of the sweep
   SweepPoint q[GCAPS_RTA_MAX_SWEEP];
 };
