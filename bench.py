@@ -40,10 +40,10 @@ LAUNCHES_PER_CALL = 9
 # grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
 # the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "40666923b4df87b626a15993f173a82490dcf20f8e7ce21a42103b36dca5c544",
+    "source_sha256": "50cd19d7d42247fcf56218982dd996a6004ba425feec48f588d8a66b6b84b74f",
     "workload": "large",
-    "bytes_per_taskset": {"gcaps": (1248194000 + 84010496) / 131072.0,
-                          "rr": (1247363000 + 83190272) / 131072.0},
+    "bytes_per_taskset": {"gcaps": (1248168000 + 84309760) / 131072.0,
+                          "rr": (1247998000 + 84658176) / 131072.0},
 }
 
 
