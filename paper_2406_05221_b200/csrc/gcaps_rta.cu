@@ -21,6 +21,11 @@
 // the warps of a launch hold the same number of tasks per lane; inside a launch warps pull chunks
 // of tasksets from a counter, because iteration counts differ widely.
 //
+// A "one warp" above is a group of 8 or 16 lanes for tasksets of up to 32 tasks (two or four
+// tasksets per warp).  gcaps_rta_multi_batch / gcaps_rta_sweep_batch use the same code with one
+// staging, ordering and aggregation per taskset and one recurrence per requested analysis and
+// (timeslice, overhead) pair.
+//
 // Everything is integer arithmetic on microseconds.  No tensor cores: nothing here is a dense
 // contraction.  No host synchronisation and no allocation in gcaps_rta_batch.
 #include <cuda_runtime.h>
@@ -446,14 +451,12 @@ struct ModeTag {
 // interferers of the task of rank `pos` sit in lanes (pos-1) % LPT downwards of slots up to
 // (pos-1) / LPT and higher slots can be skipped.
 //
-// SWEEP: the taskset is staged, ordered and aggregated once and then analysed under every
-// (timeslice, overhead) pair of `sw`; pair q writes out_wcrt + q * n_tasks (skipped when out_wcrt
-// is null) and out_sched + q * n_tasksets.
-//
-// MASK: bit m set = analysis MODE m is run.  One bit: the plain kernels.  Several bits (always
-// with SWEEP): every (timeslice, overhead) pair is analysed under each mode of MASK that
-// sw->enabled also names, in ascending mode order; the k-th analysis of a taskset writes result
-// block k (out_wcrt + k * n_tasks, out_sched + k * n_tasksets).
+// MASK: bit m set = analysis MODE m is compiled in.  SWEEP: the taskset is staged, ordered and
+// aggregated once and then analysed under every (timeslice, overhead) pair q of `sw` and every
+// mode m of MASK that sw->enabled names; that analysis writes result block
+// q * sw->block_stride + sw->block_of_mode[m] (out_wcrt + block * n_tasks, skipped when out_wcrt
+// is null; out_sched + block * n_tasksets).  Without SWEEP, MASK has one bit and the analysis
+// takes its constants and outputs from `p`.
 template <int LPT, int SLOTS, int MASK, bool SWEEP = false>
 __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane,
                                              unsigned int gmask, const SweepArgs *sw = nullptr) {
