@@ -40,10 +40,10 @@ LAUNCHES_PER_CALL = 9
 # grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
 # the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "50cd19d7d42247fcf56218982dd996a6004ba425feec48f588d8a66b6b84b74f",
+    "source_sha256": "cf7ad0323ea1b6775be2023e01304e929222710b6137042caed14493729d6486",
     "workload": "large",
-    "bytes_per_taskset": {"gcaps": (1248168000 + 84309760) / 131072.0,
-                          "rr": (1247998000 + 84658176) / 131072.0},
+    "bytes_per_taskset": {"gcaps": (1248341000 + 84559872) / 131072.0,
+                          "rr": (1247893000 + 84667904) / 131072.0},
 }
 
 
