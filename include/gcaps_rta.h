@@ -329,14 +329,16 @@ typedef struct gcaps_gen_params {
   int32_t wfd;                   /* 1: worst-fit-decreasing re-allocation of tasks to CPUs      */
 } gcaps_gen_params_t;
 
-/* Scratch of gcaps_gen_count / gcaps_gen_fill for `count` tasksets (host computation). */
-size_t gcaps_gen_workspace_bytes(int64_t count);
+/* Scratch of gcaps_gen_count / gcaps_gen_fill for `count` tasksets of these parameters (host
+ * computation; 12 bytes per possible task of a taskset plus 64 bytes per taskset; 0 for a
+ * non-positive count or parameters outside the limits). */
+size_t gcaps_gen_workspace_bytes(const gcaps_gen_params_t *params, int64_t count);
 
 /*
  * gcaps_gen_count -- sizes of tasksets first .. first+count-1 of the stream: writes their
  * offsets into `workspace` (kept for gcaps_gen_fill) and the three array lengths n_tasks,
  * n_csegs, n_gsegs to out_totals (DEVICE, 3 x int64; read them back to size the arrays).
- * workspace: DEVICE, gcaps_gen_workspace_bytes(count) bytes, 256-byte aligned.  Asynchronous on
+ * workspace: DEVICE, gcaps_gen_workspace_bytes(params, count) bytes, 256-byte aligned.  Asynchronous on
  * `stream`; GCAPS_OK or a GCAPS_ERR_* (parameters outside the limits stated above:
  * GCAPS_ERR_INVALID_ARG).
  */

@@ -101,7 +101,7 @@ def load_library(path: Optional[str] = None):
             ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int, _p64, _p64,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         lib.gcaps_rta_multi_batch.restype = ctypes.c_int
-        lib.gcaps_gen_workspace_bytes.argtypes = [ctypes.c_int64]
+        lib.gcaps_gen_workspace_bytes.argtypes = [ctypes.POINTER(IntParams), ctypes.c_int64]
         lib.gcaps_gen_workspace_bytes.restype = ctypes.c_size_t
         lib.gcaps_gen_count.argtypes = [ctypes.POINTER(IntParams), ctypes.c_int64, ctypes.c_int64,
                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
@@ -300,7 +300,8 @@ def generate_device(params: GenParams, first: int, count: int, device="cuda:0", 
     cp = params.int_params()
     with torch.cuda.device(dev):
         st = stream if stream is not None else torch.cuda.current_stream(dev)
-        ws = torch.empty(max(int(lib.gcaps_gen_workspace_bytes(count)), 256), dtype=torch.uint8, device=dev)
+        ws = torch.empty(max(int(lib.gcaps_gen_workspace_bytes(ctypes.byref(cp), count)), 256), dtype=torch.uint8,
+                         device=dev)
         totals = torch.zeros(3, dtype=torch.int64, device=dev)
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if timing is not None else None
         if ev:

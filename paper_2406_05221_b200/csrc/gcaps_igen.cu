@@ -2,10 +2,14 @@
 // GCAPS, ECRTS 2024, arXiv 2406.05221, Sec. 7.1 / Table 3) for NVIDIA B200 (sm_100a).
 //
 // The generator itself is igen.h (integer-only; the host generator compiles the same
-// definition).  Here: one thread per taskset.  gcaps_gen_count runs the per-task part of the
-// generator and writes the three sizes of every taskset, then three exclusive scans turn them
-// into offsets (block sums, one block over the block sums, block-local scan).  gcaps_gen_fill
-// runs the generator again and writes every value at its offset.
+// definition).  gcaps_gen_count: one thread per taskset runs the per-task part of the generator
+// (igen_begin), writes the three sizes of the taskset and leaves what it drew per task (period,
+// execution demand, priority, core, GPU segments: 12 bytes per task) and the position of the
+// random stream in the workspace; three exclusive scans turn the sizes into offsets (block sums,
+// one block over the block sums, block-local scan).  gcaps_gen_fill: one warp per taskset, lane =
+// task; the random draws of a task start at a position that is a prefix sum over the tasks
+// before it (the random source is counter-based), so every lane splits its own task's demand
+// into segments (igen_task_segments) and writes them at offsets that are prefix sums again.
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <string.h>
@@ -23,12 +27,21 @@ constexpr int kGenThreads = 128;
 constexpr int kScanThreads = 256;
 constexpr int kScanItems = 4 * kScanThreads;  // elements of one scan block
 
-// workspace: off[3][count + 1] (tasks, CPU segments, GPU segments), then block sums [3][blocks]
+// workspace: off[3][count + 1] (tasks, CPU segments, GPU segments), block sums [3][blocks], then
+// the per-taskset state: state_stride 32-bit words each -- key and counter of the random stream
+// (4 words), then per task T, E and (priority | core << 16 | GPU segments << 24)
 struct GenSpace {
   i64 *off[3];
   i64 *block_sum[3];
   i64 n_blocks;
+  u32 *state;
+  i64 state_stride;
 };
+
+__host__ __device__ inline i64 max_tasks_of(const igen_params_t &p) {
+  const i64 m = (i64)p.cores_hi * (i64)p.tpc_hi;
+  return m > IGEN_MAX_TASKS ? IGEN_MAX_TASKS : m;
+}
 
 __host__ __device__ inline i64 scan_blocks(i64 count) { return (count + kScanItems - 1) / kScanItems; }
 
@@ -39,6 +52,14 @@ __global__ void __launch_bounds__(kGenThreads) gen_count_kernel(igen_params_t p,
   igen_state_t s;
   igen_begin(&p, (uint64_t)(first + t), &s);
   w.off[0][t] = s.n, w.off[1][t] = s.n_csegs, w.off[2][t] = s.n_gsegs;
+  u32 *st = w.state + t * w.state_stride;
+  st[0] = (u32)s.rng.key, st[1] = (u32)(s.rng.key >> 32);
+  st[2] = (u32)s.rng.ctr, st[3] = (u32)(s.rng.ctr >> 32);
+  for (int i = 0; i < s.n; ++i) {
+    st[4 + 3 * i] = s.T[i];
+    st[5 + 3 * i] = s.E[i];
+    st[6 + 3 * i] = (u32)s.prio[i] | ((u32)s.core[i] << 16) | ((u32)s.eta[i] << 24);
+  }
 }
 
 __device__ __forceinline__ i64 block_exclusive_scan(i64 v, i64 *total, i64 *warp_sums) {
@@ -126,34 +147,60 @@ struct GenOut {
   i64 cap_tasks, cap_csegs, cap_gsegs;
 };
 
+__device__ __forceinline__ u32 warp_exclusive(u32 v, int lane, u32 *total) {
+  u32 x = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 y = __shfl_up_sync(kFull, x, d);
+    if (lane >= d) x += y;
+  }
+  *total = __shfl_sync(kFull, x, 31);
+  return x - v;
+}
+
 __global__ void __launch_bounds__(kGenThreads) gen_fill_kernel(igen_params_t p, i64 first, i64 count,
                                                                 GenSpace w, GenOut o) {
-  const i64 t = (i64)blockIdx.x * kGenThreads + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const i64 t = (i64)blockIdx.x * (kGenThreads / 32) + (threadIdx.x >> 5);
   if (t >= count) return;
-  igen_state_t s;
-  igen_begin(&p, (uint64_t)(first + t), &s);
-  const i64 k0 = w.off[0][t];
-  i64 c0 = w.off[1][t], g0 = w.off[2][t];
-  o.task_off[t] = k0;
-  const bool fits = k0 + s.n <= o.cap_tasks && c0 + s.n_csegs <= o.cap_csegs && g0 + s.n_gsegs <= o.cap_gsegs;
+  const i64 k0 = w.off[0][t], n = w.off[0][t + 1] - k0;
+  const i64 c_start = w.off[1][t], g_start = w.off[2][t];
+  if (lane == 0) o.task_off[t] = k0;
+  const bool fits = k0 + n <= o.cap_tasks && w.off[1][t + 1] <= o.cap_csegs && w.off[2][t + 1] <= o.cap_gsegs;
   if (fits) {
-    for (int i = 0; i < s.n; ++i) {
-      int64_t cs[IGEN_MAX_SEGS + 1], gm[IGEN_MAX_SEGS], ge[IGEN_MAX_SEGS];
-      igen_segments(&s, i, cs, gm, ge);
-      o.period[k0 + i] = s.T[i];
-      o.deadline[k0 + i] = s.T[i];
-      o.priority[k0 + i] = s.prio[i];
-      o.core[k0 + i] = s.core[i];
-      o.cseg_off[k0 + i] = c0;
-      o.gseg_off[k0 + i] = g0;
-      const int eta = s.eta[i];
-      for (int j = 0; j <= eta; ++j) o.cseg_wcet[c0 + j] = cs[j];
-      for (int j = 0; j < eta; ++j) o.gseg_misc[g0 + j] = gm[j], o.gseg_exec[g0 + j] = ge[j];
-      c0 += eta + 1;
-      g0 += eta;
+    const u32 *st = w.state + t * w.state_stride;
+    const uint64_t key = (uint64_t)st[0] | ((uint64_t)st[1] << 32);
+    uint64_t ctr = (uint64_t)st[2] | ((uint64_t)st[3] << 32);
+    u32 c_run = 0, g_run = 0;  // segments of the tasks before this round of 32
+    for (i64 i0 = 0; i0 < n; i0 += 32) {
+      const i64 i = i0 + lane;
+      const bool mine = i < n;
+      u32 T = 0, E = 0, pk = 0;
+      if (mine) T = st[4 + 3 * i], E = st[5 + 3 * i], pk = st[6 + 3 * i];
+      const int eta = (int)(pk >> 24);
+      u32 draws_total, c_total, g_total;
+      const u32 draws_before = warp_exclusive(mine ? igen_task_draws(eta) : 0u, lane, &draws_total);
+      const u32 c_before = warp_exclusive(mine ? (u32)eta + 1u : 0u, lane, &c_total);
+      const u32 g_before = warp_exclusive(mine ? (u32)eta : 0u, lane, &g_total);
+      if (mine) {
+        igen_rng_t rng;
+        rng.key = key, rng.ctr = ctr + draws_before;
+        int64_t cs[IGEN_MAX_SEGS + 1], gm[IGEN_MAX_SEGS], ge[IGEN_MAX_SEGS];
+        igen_task_segments(&rng, (int64_t)E, eta, p.ratio_lo, p.ratio_hi, cs, gm, ge);
+        const i64 c0 = c_start + c_run + c_before, g0 = g_start + g_run + g_before;
+        o.period[k0 + i] = T;
+        o.deadline[k0 + i] = T;
+        o.priority[k0 + i] = pk & 0xffffu;
+        o.core[k0 + i] = (pk >> 16) & 0xffu;
+        o.cseg_off[k0 + i] = c0;
+        o.gseg_off[k0 + i] = g0;
+        for (int j = 0; j <= eta; ++j) o.cseg_wcet[c0 + j] = cs[j];
+        for (int j = 0; j < eta; ++j) o.gseg_misc[g0 + j] = gm[j], o.gseg_exec[g0 + j] = ge[j];
+      }
+      ctr += draws_total, c_run += c_total, g_run += g_total;
     }
   }
-  if (t == count - 1) {
+  if (t == count - 1 && lane == 0) {
     o.task_off[count] = w.off[0][count];
     if (w.off[0][count] <= o.cap_tasks) {
       o.cseg_off[w.off[0][count]] = w.off[1][count];
@@ -175,8 +222,9 @@ bool params_ok(const gcaps_gen_params_t *p) {
          p->seg_hi >= p->seg_lo && p->seg_hi <= IGEN_MAX_SEGS;
 }
 
-int make_space(GenSpace *w, int64_t count, void *workspace, size_t workspace_bytes) {
-  if (!workspace || workspace_bytes < gcaps_gen_workspace_bytes(count) || ((uintptr_t)workspace & 255u))
+int make_space(GenSpace *w, const gcaps_gen_params_t *params, int64_t count, void *workspace,
+               size_t workspace_bytes) {
+  if (!workspace || workspace_bytes < gcaps_gen_workspace_bytes(params, count) || ((uintptr_t)workspace & 255u))
     return GCAPS_ERR_WORKSPACE;
   unsigned char *b = (unsigned char *)workspace;
   const size_t off_bytes = align256((size_t)(count + 1) * sizeof(i64));
@@ -186,6 +234,10 @@ int make_space(GenSpace *w, int64_t count, void *workspace, size_t workspace_byt
     w->off[a] = (i64 *)(b + a * off_bytes);
     w->block_sum[a] = (i64 *)(b + 3 * off_bytes + a * sum_bytes);
   }
+  igen_params_t p;
+  memcpy(&p, params, sizeof(p));
+  w->state = (u32 *)(b + 3 * off_bytes + 3 * sum_bytes);
+  w->state_stride = 4 + 3 * max_tasks_of(p);
   return GCAPS_OK;
 }
 
@@ -193,10 +245,13 @@ int make_space(GenSpace *w, int64_t count, void *workspace, size_t workspace_byt
 
 extern "C" {
 
-size_t gcaps_gen_workspace_bytes(int64_t count) {
-  if (count <= 0) return 0;
+size_t gcaps_gen_workspace_bytes(const gcaps_gen_params_t *params, int64_t count) {
+  if (count <= 0 || !params_ok(params)) return 0;
+  igen_params_t p;
+  memcpy(&p, params, sizeof(p));
   return 3 * align256((size_t)(count + 1) * sizeof(i64)) +
-         3 * align256((size_t)scan_blocks(count) * sizeof(i64));
+         3 * align256((size_t)scan_blocks(count) * sizeof(i64)) +
+         align256((size_t)count * (size_t)(4 + 3 * max_tasks_of(p)) * sizeof(u32));
 }
 
 int gcaps_gen_count(const gcaps_gen_params_t *params, int64_t first, int64_t count,
@@ -216,7 +271,7 @@ int gcaps_gen_count(const gcaps_gen_params_t *params, int64_t first, int64_t cou
     return GCAPS_OK;
   }
   GenSpace w;
-  rc = make_space(&w, count, workspace, workspace_bytes);
+  rc = make_space(&w, params, count, workspace, workspace_bytes);
   if (rc != GCAPS_OK) return rc;
   igen_params_t p;
   memcpy(&p, params, sizeof(p));
@@ -244,7 +299,7 @@ int gcaps_gen_fill(const gcaps_gen_params_t *params, int64_t first, int64_t coun
   int rc = device_info(&di);
   if (rc != GCAPS_OK) return rc;
   GenSpace w;
-  rc = make_space(&w, count, workspace, workspace_bytes);
+  rc = make_space(&w, params, count, workspace, workspace_bytes);
   if (rc != GCAPS_OK) return rc;
   igen_params_t p;
   memcpy(&p, params, sizeof(p));
@@ -254,8 +309,9 @@ int gcaps_gen_fill(const gcaps_gen_params_t *params, int64_t first, int64_t coun
   o.cseg_wcet = (i64 *)ts->cseg_wcet, o.gseg_off = (i64 *)ts->gseg_off;
   o.gseg_misc = (i64 *)ts->gseg_misc, o.gseg_exec = (i64 *)ts->gseg_exec;
   o.cap_tasks = ts->n_tasks, o.cap_csegs = ts->n_csegs, o.cap_gsegs = ts->n_gsegs;
-  gen_fill_kernel<<<(unsigned int)((count + kGenThreads - 1) / kGenThreads), kGenThreads, 0,
-                    (cudaStream_t)stream>>>(p, first, count, w, o);
+  constexpr int kWarps = kGenThreads / 32;
+  gen_fill_kernel<<<(unsigned int)((count + kWarps - 1) / kWarps), kGenThreads, 0, (cudaStream_t)stream>>>(
+      p, first, count, w, o);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;

@@ -296,25 +296,34 @@ IGEN_FN void igen_begin(const igen_params_t *p, uint64_t index, igen_state_t *s)
   }
 }
 
-/* The segments of task i (call for i = 0, 1, ... in order): cseg[0 .. eta], gm / ge[0 .. eta-1]. */
-IGEN_FN void igen_segments(igen_state_t *s, int i, int64_t *cseg, int64_t *gm, int64_t *ge) {
-  const int64_t E = s->E[i];
-  const int eta = s->eta[i];
-  const uint64_t rho = igen_range(&s->rng, s->ratio_lo, s->ratio_hi);
-  int64_t G = (int64_t)((rho * (uint64_t)E + (1ULL << 31)) >> 32); /* rho < 2^32, E < 2^24 */
+/* Random draws igen_task_segments() takes for a task with eta GPU segments: the ratio, eta
+ * weights of the GPU split (none for a CPU-only task), eta + 1 weights of the CPU split. */
+IGEN_FN uint32_t igen_task_draws(int eta) { return 2u * (uint32_t)eta + 2u; }
+
+/* The segments of a task with execution demand E and eta GPU segments, drawn from `rng`:
+ * cseg[0 .. eta], gm / ge[0 .. eta-1]. */
+IGEN_FN void igen_task_segments(igen_rng_t *rng, int64_t E, int eta, uint64_t ratio_lo,
+                                uint64_t ratio_hi, int64_t *cseg, int64_t *gm, int64_t *ge) {
+  const uint64_t rho = igen_range(rng, ratio_lo, ratio_hi);
+  int64_t G = (int64_t)((rho * (uint64_t)E + (1ULL << 31)) >> 32); /* rho < 2^32, E < 2^31 */
   if (eta == 0) {
     G = 0;
   } else {
     if (G < eta) G = eta;
     if (G > E - eta - 1) G = E - eta - 1;
     int64_t g[IGEN_MAX_SEGS];
-    igen_split(&s->rng, G, eta, g);
+    igen_split(rng, G, eta, g);
     for (int j = 0; j < eta; ++j) {
       gm[j] = g[j] / 5; /* 20 % miscellaneous CPU work, 80 % pure GPU work */
       ge[j] = g[j] - gm[j];
     }
   }
-  igen_split(&s->rng, E - G, eta + 1, cseg);
+  igen_split(rng, E - G, eta + 1, cseg);
+}
+
+/* The segments of task i of the state (call for i = 0, 1, ... in order). */
+IGEN_FN void igen_segments(igen_state_t *s, int i, int64_t *cseg, int64_t *gm, int64_t *ge) {
+  igen_task_segments(&s->rng, s->E[i], s->eta[i], s->ratio_lo, s->ratio_hi, cseg, gm, ge);
 }
 
 #endif /* GCAPS_IGEN_H_ */

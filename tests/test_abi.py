@@ -34,7 +34,11 @@ def test_host_only_entry_points(lib):
     assert binding.workspace_bytes(0) == 0 and binding.workspace_bytes(-5) == 0
     small, big = binding.workspace_bytes(1), binding.workspace_bytes(1_000_000)
     assert small >= 4 and big >= 4 * 1_000_000 and big % 256 == 0
-    assert lib.gcaps_gen_workspace_bytes(0) == 0 and lib.gcaps_gen_workspace_bytes(1000) % 256 == 0
+    from paper_2406_05221_b200 import taskgen
+    gp = taskgen.WORKLOADS["large"].streams[0].int_params()
+    assert lib.gcaps_gen_workspace_bytes(ctypes.byref(gp), 0) == 0
+    big = lib.gcaps_gen_workspace_bytes(ctypes.byref(gp), 1000)
+    assert big % 256 == 0 and big >= 1000 * (4 + 3 * 80) * 4
     for code in (0, -1, -2, -3, -4, -99):
         assert lib.gcaps_rta_strerror(code)
 

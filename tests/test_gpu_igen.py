@@ -82,7 +82,7 @@ def test_empty_and_argument_errors():
     lib = binding.load_library()
     good = w.streams[0].int_params()
     totals = torch.zeros(3, dtype=torch.int64, device="cuda")
-    ws = torch.empty(int(lib.gcaps_gen_workspace_bytes(100)), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(int(lib.gcaps_gen_workspace_bytes(ctypes.byref(good), 100)), dtype=torch.uint8, device="cuda")
     bad = w.streams[0].int_params()
     bad.tpc_hi = 300
     assert lib.gcaps_gen_count(ctypes.byref(bad), 0, 100, totals.data_ptr(), ws.data_ptr(), ws.numel(), None) == binding.ERR_INVALID_ARG
@@ -102,7 +102,7 @@ def test_arrays_that_are_too_short_are_not_overrun():
     cp = w.streams[0].int_params()
     count = 500
     twin = w.generate(0, count, integer=True)
-    ws = torch.empty(int(lib.gcaps_gen_workspace_bytes(count)), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(int(lib.gcaps_gen_workspace_bytes(ctypes.byref(cp), count)), dtype=torch.uint8, device="cuda")
     totals = torch.zeros(3, dtype=torch.int64, device="cuda")
     assert lib.gcaps_gen_count(ctypes.byref(cp), 0, count, totals.data_ptr(), ws.data_ptr(), ws.numel(), None) == 0
     assert totals.cpu().tolist() == [twin.n_tasks, twin.n_csegs, twin.n_gsegs]
