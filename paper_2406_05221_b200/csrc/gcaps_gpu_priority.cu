@@ -39,8 +39,20 @@ struct GpSmem {
   short gpu_rank[MAXN];     // the same for the given GPU priorities
   short by_cpu_rank[MAXN];  // CPU rank -> position
   unsigned char uses_gpu[MAXN];
-  unsigned char placed[MAXN];  // search: the task has its level
+  // search: bit r set = the task of CPU rank r has no level yet and no task of lower CPU priority
+  // on its core is without one, i.e. it may take the next level (the same-core rule of Sec. 5.3)
+  unsigned int cand[8];
 };
+
+// Largest r < below with bit r set in the 256-bit set `bits`, or -1.
+__device__ __forceinline__ int highest_below(const unsigned int *bits, int below) {
+  for (int w = (below - 1) >> 5; w >= 0; --w) {
+    unsigned int m = bits[w];
+    if (w == (below - 1) >> 5) m &= (2u << ((below - 1) & 31)) - 1u;  // (2u << 31 wraps to 0: all ones)
+    if (m) return 32 * w + 31 - __clz((int)m);
+  }
+  return -1;
+}
 
 // What a lane knows about its S tasks as interferers (slot s: position lane + LPT * s).
 template <int S>
@@ -289,37 +301,57 @@ __device__ void analyse_gpu_priority(const GpParams &g, i64 t, GpSmem<LPT * S> &
   } else {
     // ---- the search of Sec. 5.3: levels from the lowest ----------------------------------------
     bool unplaced[S];
+    if (lane < 8) sm.cand[lane] = 0;
 #pragma unroll
     for (int s = 0; s < S; ++s) {
       unplaced[s] = valid[s];
       if (valid[s]) {
-        sm.placed[lane + LPT * s] = 0;
         p.out_wcrt[a + lane + LPT * s] = GCAPS_WCRT_MISS;
         g.gpu_prio_out[a + lane + LPT * s] = 0;
       }
     }
     __syncwarp(gmask);
+#pragma unroll
+    for (int s = 0; s < S; ++s) {  // the lowest CPU priority of every core starts as a candidate
+      if (valid[s]) {
+        bool lowest = true;
+        for (int q = 0; q < n; ++q) lowest &= !(sm.core[q] == core[s] && sm.cpu_rank[q] > me.cpu_rank[s]);
+        if (lowest) atomicOr(&sm.cand[me.cpu_rank[s] >> 5], 1u << (me.cpu_rank[s] & 31));
+      }
+    }
+    __syncwarp(gmask);
     for (int level = 1; level <= n && sched == GCAPS_SCHED_YES; ++level) {
       bool placed = false;
-      for (int want = n - 1; want >= 0 && !placed; --want) {  // lowest CPU priority first
+      int want = n;
+      while (!placed) {  // candidates from the lowest CPU priority upwards
+        want = highest_below(sm.cand, want);
+        if (want < 0) break;
         const int c = sm.by_cpu_rank[want];
-        if (sm.placed[c]) continue;
-        const int core_c = sm.core[c];
-        bool lower = false;  // an unplaced task of lower CPU priority on the same core bars c
-#pragma unroll
-        for (int s = 0; s < S; ++s) lower |= unplaced[s] && core[s] == core_c && me.cpu_rank[s] > want;
-        if (__any_sync(gmask, lower)) continue;
         const i64 r = bound(c, unplaced);  // every other unplaced task above c (c itself is skipped)
         if (r >= 0) {
           placed = true;
+          const int core_c = sm.core[c];
+          int next = -1;  // the task of c's core that becomes a candidate now
 #pragma unroll
-          for (int s = 0; s < S; ++s)
+          for (int s = 0; s < S; ++s) {
             if (lane + LPT * s == c) {
               unplaced[s] = false;
-              sm.placed[c] = 1;
               p.out_wcrt[a + c] = r;
               g.gpu_prio_out[a + c] = (i64)level;
             }
+            if (unplaced[s] && core[s] == core_c && me.cpu_rank[s] < want && me.cpu_rank[s] > next)
+              next = me.cpu_rank[s];
+          }
+#pragma unroll
+          for (int d = LPT / 2; d >= 1; d >>= 1) {
+            const int other = __shfl_xor_sync(gmask, next, d, LPT);
+            next = other > next ? other : next;
+          }
+          __syncwarp(gmask);
+          if (lane == 0) {
+            sm.cand[want >> 5] &= ~(1u << (want & 31));
+            if (next >= 0) sm.cand[next >> 5] |= 1u << (next & 31);
+          }
           __syncwarp(gmask);
         }
       }
