@@ -346,11 +346,13 @@ int gcaps_gen_count(const gcaps_gen_params_t *params, int64_t first, int64_t cou
                     int64_t *out_totals, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * gcaps_gen_fill -- writes the tasksets whose offsets gcaps_gen_count (same params, first, count,
- * workspace) left in `workspace` into the DEVICE arrays of `ts` (ts->n_tasks, n_csegs, n_gsegs
- * state how many elements the arrays hold; a taskset that would not fit is left out and
- * GCAPS_ERR_TOO_LARGE is NOT reported asynchronously -- size the arrays from out_totals).
- * D_i = T_i.  Asynchronous on `stream`.
+ * gcaps_gen_fill -- writes the tasksets that gcaps_gen_count (same params, first, count and
+ * workspace; the workspace must be untouched in between) sized into the DEVICE arrays of `ts`.
+ * ts->n_tasks, n_csegs, n_gsegs state how many elements the caller's arrays hold: size them from
+ * out_totals.  A taskset that would reach beyond one of them is left out (its task_off entry is
+ * still written); the call cannot report that, being asynchronous.  task_off gets count + 1
+ * entries, cseg_off and gseg_off one entry more than there are tasks.  D_i = T_i.  Asynchronous on
+ * `stream`; GCAPS_OK or a GCAPS_ERR_*.
  */
 int gcaps_gen_fill(const gcaps_gen_params_t *params, int64_t first, int64_t count,
                    const gcaps_tasksets_t *ts, void *workspace, size_t workspace_bytes,
