@@ -1106,6 +1106,8 @@ constexpr int kSmallWarpWords =
 template <int MODE>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(3)) rta_small_kernel(KParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
+  asm volatile("griddepcontrol.launch_dependents;");
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
   run_bin<16, 2, 1 << MODE>(p, 3, warp_buf, ahead);
@@ -1118,6 +1120,8 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(3)) rta_small_kernel
 template <int SLOTS, int MODE>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kernel(KParams p, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
+  asm volatile("griddepcontrol.launch_dependents;");
   constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
@@ -1130,6 +1134,8 @@ template <int MASK>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(3))
 rta_small_sweep_kernel(KParams p, const __grid_constant__ SweepArgs sw) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
+  asm volatile("griddepcontrol.launch_dependents;");
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
   run_bin<16, 2, MASK, true>(p, 3, warp_buf, ahead, &sw);
@@ -1142,6 +1148,8 @@ template <int SLOTS, int MASK>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS))
 rta_big_sweep_kernel(KParams p, int bin, const __grid_constant__ SweepArgs sw) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
+  asm volatile("griddepcontrol.launch_dependents;");
   constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
@@ -1296,7 +1304,7 @@ cudaError_t launch_big(const KParams &p, int bin, int sm_count, cudaStream_t st)
   constexpr int kWarps = kBlockThreads / 32;
   static int blocks_per_sm[64] = {0};
   const size_t smem = sizeof(u32) * (bin_warp_words<32, SLOTS>() + kAheadWords) * kWarps;
-  return launch_persistent(rta_big_kernel<SLOTS, MODE>, blocks_per_sm, smem,
+  return launch_persistent_ex(true, rta_big_kernel<SLOTS, MODE>, blocks_per_sm, smem,
                            (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p, bin);
 }
 
@@ -1320,7 +1328,7 @@ cudaError_t launch_big_sweep(const KParams &p, const SweepArgs &sw, int bin, int
   constexpr int kWarps = kBlockThreads / 32;
   static int blocks_per_sm[64] = {0};
   const size_t smem = sizeof(u32) * (bin_warp_words<32, SLOTS>() + kAheadWords) * kWarps;
-  return launch_persistent(rta_big_sweep_kernel<SLOTS, MASK>, blocks_per_sm, smem,
+  return launch_persistent_ex(true, rta_big_sweep_kernel<SLOTS, MASK>, blocks_per_sm, smem,
                            (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p, bin, sw);
 }
 

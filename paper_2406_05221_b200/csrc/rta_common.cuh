@@ -148,9 +148,13 @@ __host__ __device__ __forceinline__ void make_reciprocal(u32 d, u32 &magic, u32 
 
 // Launches `kernel` (a persistent kernel of kBlockThreads threads needing `smem` bytes) with as
 // many blocks as the device keeps resident, but never more than the batch could feed.
+// overlap_previous: the kernel launched just before on this stream works on other data (another
+// size bin) and has let its dependents go (griddepcontrol.launch_dependents), so this one is
+// launched with programmatic stream serialisation and fills the SMs as that one's blocks leave
+// instead of waiting for its last block.  It needs nothing that kernel writes.
 template <typename... Args>
-cudaError_t launch_persistent(void (*kernel)(Args...), int *blocks_per_sm, size_t smem, long long want,
-                              int sm_count, cudaStream_t st, Args... args) {
+cudaError_t launch_persistent_ex(bool overlap_previous, void (*kernel)(Args...), int *blocks_per_sm,
+                                 size_t smem, long long want, int sm_count, cudaStream_t st, Args... args) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -166,8 +170,24 @@ cudaError_t launch_persistent(void (*kernel)(Args...), int *blocks_per_sm, size_
   long long grid = (long long)sm_count * blocks_per_sm[dev];
   if (grid > want) grid = want;
   if (grid < 1) grid = 1;
-  kernel<<<(unsigned int)grid, kBlockThreads, smem, st>>>(args...);
-  return cudaGetLastError();
+  if (!overlap_previous) {
+    kernel<<<(unsigned int)grid, kBlockThreads, smem, st>>>(args...);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned int)grid), cfg.blockDim = dim3(kBlockThreads);
+  cfg.dynamicSmemBytes = smem, cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr, cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+template <typename... Args>
+cudaError_t launch_persistent(void (*kernel)(Args...), int *blocks_per_sm, size_t smem, long long want,
+                              int sm_count, cudaStream_t st, Args... args) {
+  return launch_persistent_ex(false, kernel, blocks_per_sm, smem, want, sm_count, st, args...);
 }
 
 
