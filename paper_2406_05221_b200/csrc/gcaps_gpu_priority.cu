@@ -397,6 +397,8 @@ static_assert(kSmallWarpBytes % 16 == 0, "every warp's area starts 16-byte align
 // the four bins of up to 32 tasks: (lanes per taskset, tasks per lane) as in the default analysis
 __global__ void __launch_bounds__(kBlockThreads) gpu_priority_small_kernel(GpParams g) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
+  asm volatile("griddepcontrol.launch_dependents;");
   unsigned char *mine = smem_raw + (threadIdx.x >> 5) * kSmallWarpBytes;
   run_bin<16, 2>(g, 3, mine);
   run_bin<8, 3>(g, 2, mine);
@@ -408,6 +410,7 @@ __global__ void __launch_bounds__(kBlockThreads) gpu_priority_small_kernel(GpPar
 template <int S>
 __global__ void __launch_bounds__(kBlockThreads) gpu_priority_big_kernel(GpParams g, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  asm volatile("griddepcontrol.launch_dependents;");
   run_bin<32, S>(g, bin, smem_raw + (threadIdx.x >> 5) * warp_bytes<32, S>());
 }
 
@@ -415,7 +418,7 @@ template <int S>
 cudaError_t launch_big(const GpParams &g, int bin, int sm_count, cudaStream_t st) {
   constexpr int kWarps = kBlockThreads / 32;
   static int blocks_per_sm[64] = {0};
-  return launch_persistent(gpu_priority_big_kernel<S>, blocks_per_sm, warp_bytes<32, S>() * kWarps,
+  return launch_persistent_ex(true, gpu_priority_big_kernel<S>, blocks_per_sm, warp_bytes<32, S>() * kWarps,
                            (g.k.n_tasksets + kWarps - 1) / kWarps, sm_count, st, g, bin);
 }
 
