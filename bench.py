@@ -200,6 +200,8 @@ def main():
                          "followed by the GPU-priority search of the paper's Sec. 5.3 on the same batch; "
                          "sweep: all (timeslice, overhead) pairs of the workload, once as one fused "
                          "gcaps_rta_sweep_batch call and once as one gcaps_rta_batch call per pair")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay each call from a CUDA graph instead of enqueueing its launches again")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -275,6 +277,9 @@ def main():
         multi_sched = torch.empty((1, 2, ts.n_tasksets), dtype=torch.uint8, device=dev)
     L, ovh = workload.timeslice_us, workload.overhead_us
     stream = torch.cuda.current_stream(dev)
+    if args.graph:  # the legacy default stream cannot be captured
+        torch.cuda.synchronize(dev)
+        stream = torch.cuda.Stream(dev)
 
     if args.mode == "assign":
         policies, names = [binding.POLICY_GCAPS, binding.ASSIGN], ["gcaps", "gpu_priority_search"]
@@ -292,27 +297,49 @@ def main():
         sweep_wcrt = torch.empty((len(pairs), ts.n_tasks), dtype=torch.int64, device=dev)
         args.no_e2e = True
 
+    def call(k, policy):
+        if args.mode == "assign" and k == 1:
+            binding.rta_gpu_priority(ts, binding.ASSIGN, ovh, None, workspace=workspace, stream=stream)
+        elif fused:
+            binding.rta_multi(ts, binding.GCAPS_SUSPEND | binding.RR_SUSPEND, [L], [ovh],
+                              out_wcrt=multi_wcrt, out_sched=multi_sched, workspace=workspace,
+                              stream=stream)
+        elif args.mode == "sweep" and k == 0:
+            binding.rta_sweep(ts, sweep_policy, [a for a, _ in pairs], [b for _, b in pairs],
+                              out_wcrt=sweep_wcrt, out_sched=sweep_sched, workspace=workspace,
+                              stream=stream)
+        elif args.mode == "sweep":
+            for q, (a, b) in enumerate(pairs):
+                binding.rta_batch(ts, sweep_policy, a, b, out_wcrt=sweep_wcrt[q],
+                                  out_sched=sweep_sched[q], workspace=workspace, stream=stream)
+        else:
+            binding.rta_batch(ts, policy, L, ovh, out_wcrt=out_wcrt, out_sched=out_sched,
+                              workspace=workspace, stream=stream)
+
+    # --graph: each call's launches (plan kernels + one kernel per size bin) recorded once in a
+    # CUDA graph and replayed; the entry points only enqueue work on the stream they are given, so
+    # they can be captured as they are (after one plain call, which sets the kernels' attributes)
+    graphs = None
+    if args.graph:
+        for k, policy in enumerate(policies):
+            call(k, policy)
+        torch.cuda.synchronize(dev)
+        graphs = []
+        for k, policy in enumerate(policies):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                call(k, policy)
+            graphs.append(g)
+
     def step(events=None):
         for k, policy in enumerate(policies):
             if events is not None:
                 events[k].record(stream)
-            if args.mode == "assign" and k == 1:
-                binding.rta_gpu_priority(ts, binding.ASSIGN, ovh, None, workspace=workspace, stream=stream)
-            elif fused:
-                binding.rta_multi(ts, binding.GCAPS_SUSPEND | binding.RR_SUSPEND, [L], [ovh],
-                                  out_wcrt=multi_wcrt, out_sched=multi_sched, workspace=workspace,
-                                  stream=stream)
-            elif args.mode == "sweep" and k == 0:
-                binding.rta_sweep(ts, sweep_policy, [a for a, _ in pairs], [b for _, b in pairs],
-                                  out_wcrt=sweep_wcrt, out_sched=sweep_sched, workspace=workspace,
-                                  stream=stream)
-            elif args.mode == "sweep":
-                for q, (a, b) in enumerate(pairs):
-                    binding.rta_batch(ts, sweep_policy, a, b, out_wcrt=sweep_wcrt[q],
-                                      out_sched=sweep_sched[q], workspace=workspace, stream=stream)
+            if graphs is not None:
+                with torch.cuda.stream(stream):
+                    graphs[k].replay()
             else:
-                binding.rta_batch(ts, policy, L, ovh, out_wcrt=out_wcrt, out_sched=out_sched,
-                                  workspace=workspace, stream=stream)
+                call(k, policy)
         if events is not None:
             events[len(policies)].record(stream)
 
@@ -424,6 +451,7 @@ def main():
                        "timeslice_us": L, "overhead_us": ovh,
                        "analyses_per_taskset_per_step": len(pairs) if pairs else analyses_per_step,
                        "calls_per_step": len(policies),
+                       "launch": "cuda graph replay per call" if args.graph else "stream launches",
                        "sweep_pairs": pairs, "generation": generation,
                        "l2": "inputs (%.2f GB per call) against a 126 MB L2; no flush between steps"
                              % (batch.input_bytes() / 1e9),
