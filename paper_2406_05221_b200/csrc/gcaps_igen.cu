@@ -185,17 +185,16 @@ __global__ void __launch_bounds__(kGenThreads) gen_fill_kernel(igen_params_t p, 
       if (mine) {
         igen_rng_t rng;
         rng.key = key, rng.ctr = ctr + draws_before;
-        int64_t cs[IGEN_MAX_SEGS + 1], gm[IGEN_MAX_SEGS], ge[IGEN_MAX_SEGS];
-        igen_task_segments(&rng, (int64_t)E, eta, p.ratio_lo, p.ratio_hi, cs, gm, ge);
         const i64 c0 = c_start + c_run + c_before, g0 = g_start + g_run + g_before;
+        // the segment values go straight to their places in the output arrays
+        igen_task_segments(&rng, (int64_t)E, eta, p.ratio_lo, p.ratio_hi, (int64_t *)(o.cseg_wcet + c0),
+                           (int64_t *)(o.gseg_misc + g0), (int64_t *)(o.gseg_exec + g0));
         o.period[k0 + i] = T;
         o.deadline[k0 + i] = T;
         o.priority[k0 + i] = pk & 0xffffu;
         o.core[k0 + i] = (pk >> 16) & 0xffu;
         o.cseg_off[k0 + i] = c0;
         o.gseg_off[k0 + i] = g0;
-        for (int j = 0; j <= eta; ++j) o.cseg_wcet[c0 + j] = cs[j];
-        for (int j = 0; j < eta; ++j) o.gseg_misc[g0 + j] = gm[j], o.gseg_exec[g0 + j] = ge[j];
       }
       ctr += draws_total, c_run += c_total, g_run += g_total;
     }

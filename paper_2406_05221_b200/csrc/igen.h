@@ -158,26 +158,60 @@ IGEN_FN uint64_t igen_exp2(uint64_t y) {
   return ((r >> (61 - k)) + 1) >> 1;
 }
 
-/* Splits `total` into `parts` integers >= 1 (needs total >= parts) in proportion to random
- * weights in [1,2); the last part takes the rounding remainder. */
-IGEN_FN void igen_split(igen_rng_t *r, int64_t total, int parts, int64_t *out) {
-  uint64_t w[IGEN_MAX_SEGS + 1], ws = 0;
-  for (int j = 0; j < parts; ++j) {
-    w[j] = (1ULL << 32) + igen_unit(r);
-    ws += w[j];
+/* floor(a / d) for 0 < d < 2^40 and a < 2^63 */
+IGEN_FN uint64_t igen_div(uint64_t a, uint64_t d) {
+#ifdef __CUDA_ARCH__
+  /* no 64-bit division: two single-precision estimates, the second of what the first left over,
+   * then the remainder settles the quotient exactly (differences are taken modulo 2^64 and read
+   * as signed: the true ones are far below 2^63) */
+  const float inv = 1.0f / (float)d;
+  uint64_t q = (uint64_t)((float)a * inv);
+  int64_t rem = (int64_t)(a - q * d);
+  const int64_t q2 = (int64_t)((float)rem * inv);
+  q += (uint64_t)q2;
+  rem -= q2 * (int64_t)d;
+  while (rem < 0) {
+    rem += (int64_t)d;
+    q -= 1;
   }
-  const uint64_t spare = (uint64_t)(total - parts); /* < 2^24: spare * w stays inside 64 bits */
+  while (rem >= (int64_t)d) {
+    rem -= (int64_t)d;
+    q += 1;
+  }
+  return q;
+#else
+  return a / d;
+#endif
+}
+
+/* Splits `total` into `parts` integers >= 1 (needs total >= parts) in proportion to random
+ * weights in [1,2); the last part takes the rounding remainder.  With `fifth` given, a fifth of
+ * every part (rounded down) goes there and the rest to `out`.  The weights are drawn twice (once
+ * for their sum, once to use them: the random source is counter-based) instead of being kept. */
+IGEN_FN void igen_split(igen_rng_t *r, int64_t total, int parts, int64_t *out, int64_t *fifth) {
+  const uint64_t first_draw = r->ctr;
+  uint64_t ws = 0;
+  for (int j = 0; j < parts; ++j) ws += (1ULL << 32) + igen_unit(r);
+  r->ctr = first_draw;
+  const uint64_t spare = (uint64_t)(total - parts); /* < 2^30: spare * w stays inside 63 bits */
   uint64_t used = 0;
   for (int j = 0; j < parts; ++j) {
+    const uint64_t w = (1ULL << 32) + igen_unit(r);
     uint64_t x;
     if (j == parts - 1) {
       x = spare - used;
     } else {
-      x = spare * w[j] / ws;
+      x = igen_div(spare * w, ws);
       if (x > spare - used) x = spare - used;
     }
     used += x;
-    out[j] = 1 + (int64_t)x;
+    const int64_t part = 1 + (int64_t)x;
+    if (fifth) {
+      fifth[j] = part / 5;
+      out[j] = part - part / 5;
+    } else {
+      out[j] = part;
+    }
   }
 }
 
@@ -311,14 +345,9 @@ IGEN_FN void igen_task_segments(igen_rng_t *rng, int64_t E, int eta, uint64_t ra
   } else {
     if (G < eta) G = eta;
     if (G > E - eta - 1) G = E - eta - 1;
-    int64_t g[IGEN_MAX_SEGS];
-    igen_split(rng, G, eta, g);
-    for (int j = 0; j < eta; ++j) {
-      gm[j] = g[j] / 5; /* 20 % miscellaneous CPU work, 80 % pure GPU work */
-      ge[j] = g[j] - gm[j];
-    }
+    igen_split(rng, G, eta, ge, gm); /* 20 % miscellaneous CPU work, 80 % pure GPU work */
   }
-  igen_split(rng, E - G, eta + 1, cseg);
+  igen_split(rng, E - G, eta + 1, cseg, 0);
 }
 
 /* The segments of task i of the state (call for i = 0, 1, ... in order). */
