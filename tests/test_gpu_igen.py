@@ -37,6 +37,28 @@ def test_device_generation_equals_host_generation(name, stream, first, count):
     assert_same(ts, w.generate(first, count, stream=stream, integer=True), name)
 
 
+def test_device_generation_at_the_ends_of_the_parameter_ranges():
+    """Periods up to 2^30 us with most of a core's utilisation in one or two tasks (quotients of
+    the segment split near 2^29), up to 16 segments, harmonic periods, per-task segment counts,
+    worst-fit allocation over many cores, cores without tasks."""
+    cases = [
+        taskgen.GenParams(seed=41, cores=(1, 3), tasks_per_core=(1, 2), util_per_core=(0.9, 0.99),
+                          period_us=(5e8, 1.07e9), gpu_frac=1.0, gpu_segments=(1, 16), gpu_ratio=(0.5, 0.95)),
+        taskgen.GenParams(seed=42, cores=(1, 3), tasks_per_core=(1, 3), util_per_core=(0.5, 0.99),
+                          period_us=(1e6, 1.07e9), gpu_mode=1, gpu_segments=(0, 16), gpu_ratio=(0.0, 0.99),
+                          harmonic_frac=0.5, wfd=True),
+        taskgen.GenParams(seed=43, cores=(33, 64), tasks_per_core=(0, 4), util_per_core=(0.01, 0.2),
+                          period_us=(1.0, 50.0), gpu_frac=0.7, gpu_segments=(2, 9), gpu_ratio=(0.3, 0.9), wfd=True),
+    ]
+    for k, params in enumerate(cases):
+        ts = binding.generate_device(params, 3, 3000)
+        torch.cuda.synchronize()
+        twin = taskgen.generate(params, 3, 3000, integer=True)
+        assert_same(ts, twin, "case %d" % k)
+        if k == 0:
+            assert twin.cseg_wcet.max() > 1 << 26 and twin.gseg_exec.max() > 1 << 26
+
+
 def test_analysis_of_device_generated_tasksets():
     for name, count in (("sweep", 3000), ("large", 800), ("divergence", 2500)):
         w = taskgen.WORKLOADS[name]
