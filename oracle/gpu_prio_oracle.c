@@ -16,7 +16,7 @@
  * the level.  The order of GPU priorities of tasks on one core must equal their CPU order, so a
  * task is only a candidate while no task of lower CPU priority on its core is unassigned.
  *
- * Readings of this build (parity unpinned beyond the paper's Table 2 verdicts): tasks without GPU
+ * Readings taken where the paper is silent (parity unpinned beyond the paper's Table 2 verdicts): tasks without GPU
  * segments take part in the assignment like any other; every task gets its own outcome (bound,
  * MISS or ITER_LIMIT; nothing is SKIPPED because nothing depends on an earlier task); when the
  * assignment fails at some level the tasks still unassigned get MISS and GPU priority 0; given
