@@ -40,10 +40,10 @@ LAUNCHES_PER_CALL = 9
 # grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
 # the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "a4fa1d30b7715046b630c95efc3eeb21c021a3f6ee17aa2aa6f5c62d6d42573c",
+    "source_sha256": "c449ba471c28a7216a2c6b05de862c3fc185155dc1a52933f6f1c26c82ee6d47",
     "workload": "large",
-    "bytes_per_taskset": {"gcaps": (1248175000 + 84576512) / 131072.0,
-                          "rr": (1247953000 + 83947008) / 131072.0},
+    "bytes_per_taskset": {"gcaps": (1248705000 + 84085248) / 131072.0,
+                          "rr": (1247744000 + 84287232) / 131072.0},
 }
 
 

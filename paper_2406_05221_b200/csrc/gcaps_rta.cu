@@ -463,7 +463,11 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   typedef FastLayout<LPT, SLOTS> Lay;
   constexpr int kLog = LPT == 32 ? 5 : LPT == 16 ? 4 : 3;  // log2 of the lanes per taskset
   constexpr int MAXN = Lay::MAXN, CAP = Lay::CAP;
-  constexpr int BC = SLOTS <= 2 ? SLOTS : 2;  // prefix blocks whose loads are issued together
+  // prefix blocks of the CPU segments whose loads are issued together.  Tasksets of 65..96 tasks
+  // with a few GPU segments per task have 200..400 CPU segments: three blocks of 128 cover them
+  // in one step where two need a second, mostly empty one (80-task tasksets: -4 % for a GCAPS
+  // kernel; the RR kernels, which carry the slice sums too, lose as much to the registers it takes)
+  constexpr int BC = SLOTS <= 2 ? SLOTS : ((SLOTS == 3 && (MASK & 12) == 0 && !SWEEP) ? 3 : 2);
   constexpr int BG = 1;
   constexpr bool kAnyGcaps = (MASK & 3) != 0;
   constexpr bool kMulti = (MASK & (MASK - 1)) != 0;
