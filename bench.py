@@ -34,16 +34,17 @@ ALU_PEAK_LANEOPS = 148 * 128 * 1.965e9
 K_TERM, K_SETUP = 6, 16   # algorithmic integer lane-operations per interference term / per task
 # kernels launched by one gcaps_rta_batch call: 3 plan kernels, one analysis kernel for the bins
 # of up to 32 tasks and one each for the 64-, 96-, 128-, 192- and 256-task bins
-LAUNCHES_PER_CALL = 9
+LAUNCHES_PER_CALL = 9        # three plan kernels + one kernel per group of size bins
+LAUNCHES_PER_SMALL_CALL = 7  # batches of up to 8,192 tasksets: one plan kernel
 # DRAM bytes (read + write) per taskset of the analysis kernel on the 'large' workload, from the
 # ncu capture summarised in profiles/rta_kernel_large_131072_full.md (131,072 tasksets; traffic
 # grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
 # the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "c449ba471c28a7216a2c6b05de862c3fc185155dc1a52933f6f1c26c82ee6d47",
+    "source_sha256": "992c86b02973be248905087f74519284979b90198204ab7a2bd867e3b67426d8",
     "workload": "large",
-    "bytes_per_taskset": {"gcaps": (1248705000 + 84085248) / 131072.0,
-                          "rr": (1247744000 + 84287232) / 131072.0},
+    "bytes_per_taskset": {"gcaps": (1248971000 + 84039424) / 131072.0,
+                          "rr": (1247874000 + 84161792) / 131072.0},
 }
 
 
@@ -458,9 +459,9 @@ def main():
                        "schedulable_fraction_last_policy": sched_frac,
                        "input_checksum": batch.checksum() if count <= 200_000 else None},
             "clocks": clocks, "e2e": e2e,
-            "gpu_launches": args.steps * (len(policies) * LAUNCHES_PER_CALL if args.mode == "policies"
-                                          else (1 + len(pairs)) * LAUNCHES_PER_CALL if args.mode == "sweep"
-                                          else 2 * LAUNCHES_PER_CALL),
+            "gpu_launches": args.steps * (len(policies) if args.mode == "policies"
+                                          else (1 + len(pairs)) if args.mode == "sweep" else 2)
+                            * (LAUNCHES_PER_SMALL_CALL if count <= 8192 else LAUNCHES_PER_CALL),
             "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
         }
         print(json.dumps(line))

@@ -106,6 +106,33 @@ __global__ void plan_scatter_kernel(KParams p) {
   }
 }
 
+// The three steps in one block, for batches small enough that launches cost more than the work.
+__global__ void __launch_bounds__(1024) plan_small_kernel(KParams p) {
+  __shared__ unsigned int cnt[kBinStride], start[kBinStride];
+  if (threadIdx.x < kBinStride) cnt[threadIdx.x] = 0;
+  __syncthreads();
+  for (i64 t = threadIdx.x; t < p.n_tasksets; t += blockDim.x)
+    atomicAdd(&cnt[size_bin(p.task_off[t + 1] - p.task_off[t])], 1u);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned int s = 0;
+    for (int k = 0; k < kBinStride; ++k) {
+      const unsigned int c = k < kNumBins ? cnt[k] : 0u;
+      p.hdr->bin_start[k] = s;
+      p.hdr->bin_count[k] = c;
+      p.hdr->next[k] = 0;
+      start[k] = s;
+      cnt[k] = 0;  // from here on the write cursor of the bin
+      s += c;
+    }
+  }
+  __syncthreads();
+  for (i64 t = threadIdx.x; t < p.n_tasksets; t += blockDim.x) {
+    const int b = size_bin(p.task_off[t + 1] - p.task_off[t]);
+    p.perm[start[b] + atomicAdd(&cnt[b], 1u)] = (unsigned int)t;
+  }
+}
+
 // Shared-memory image of one taskset, indexed by priority rank unless noted.
 template <int MAXN>
 struct GroupSmem {
@@ -1293,6 +1320,10 @@ int enqueue_plan(KParams &p, void *workspace, size_t workspace_bytes, cudaStream
   p.hdr = (PlanHeader *)w;
   p.block_cnt = (unsigned int *)(w + 256);
   p.perm = (unsigned int *)(w + 256 + align_up(nb * kBinStride * sizeof(unsigned int), 256));
+  if (p.n_tasksets <= kPlanSmall) {
+    plan_small_kernel<<<1, 1024, 0, st>>>(p);
+    return GCAPS_OK;
+  }
   plan_count_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);
   plan_scan_kernel<<<1, 32 * kNumBins, 0, st>>>(p, (unsigned int)nb);
   plan_scatter_kernel<<<(unsigned int)nb, 256, 0, st>>>(p);

@@ -22,6 +22,7 @@ constexpr u32 kFastLimit = 1u << 26;  // fast path: every time of the taskset is
 constexpr u32 kFastClamp = 1u << 26;  // ... so a sum clamped here still exceeds every deadline
 constexpr int kBlockThreads = 128;
 constexpr int kPlanItems = 1024;  // tasksets per plan block
+constexpr int kPlanSmall = 8192;  // batches up to this size are planned by one block in one launch
 constexpr u64 kClamp = 1ull << 50;  // any quantity >= 2^50 exceeds every deadline (<= 2^40)
 
 struct PlanHeader {
