@@ -211,15 +211,47 @@ __device__ void analyse_gpu_priority(const GpParams &g, i64 t, GpSmem<LPT * S> &
   }
   // ---- CPU ranks: larger priority first, ties by position -----------------------------------
   GpLane<S> me;
+  // distinct priorities hi-n+1 .. hi (what a numbering by period gives): the rank is hi - priority
+  i64 hi = INT64_MIN;
+#pragma unroll
+  for (int s = 0; s < S; ++s)
+    if (valid[s] && sm.key[lane + LPT * s] > hi) hi = sm.key[lane + LPT * s];
+#pragma unroll
+  for (int d = LPT / 2; d >= 1; d >>= 1) {
+    const i64 other = __shfl_xor_sync(gmask, hi, d, LPT);
+    hi = other > hi ? other : hi;
+  }
+  bool dense = true;
 #pragma unroll
   for (int s = 0; s < S; ++s) {
-    const int i = lane + LPT * s;
-    int r = 0;
-    if (valid[s]) {
-      const i64 pi = sm.key[i];
-      for (int q = 0; q < n; ++q) r += (sm.key[q] > pi || (sm.key[q] == pi && q < i)) ? 1 : 0;
+    const u64 r = valid[s] ? (u64)hi - (u64)sm.key[lane + LPT * s] : 0;
+    dense &= r < (u64)n;
+    me.cpu_rank[s] = (int)(r < (u64)n ? r : 0);
+  }
+  dense = __all_sync(gmask, dense);
+  if (dense) {  // ... and no rank taken twice
+#pragma unroll
+    for (int s = 0; s < S; ++s)
+      if (valid[s]) sm.by_cpu_rank[me.cpu_rank[s]] = (short)(lane + LPT * s);
+    __syncwarp(gmask);
+    bool uniq = true;
+#pragma unroll
+    for (int s = 0; s < S; ++s)
+      if (valid[s]) uniq &= sm.by_cpu_rank[me.cpu_rank[s]] == (short)(lane + LPT * s);
+    dense = __all_sync(gmask, uniq);
+    __syncwarp(gmask);
+  }
+  if (!dense) {  // any priorities: count the tasks that come before
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+      const int i = lane + LPT * s;
+      int r = 0;
+      if (valid[s]) {
+        const i64 pi = sm.key[i];
+        for (int q = 0; q < n; ++q) r += (sm.key[q] > pi || (sm.key[q] == pi && q < i)) ? 1 : 0;
+      }
+      me.cpu_rank[s] = r;
     }
-    me.cpu_rank[s] = r;
   }
   __syncwarp(gmask);
 #pragma unroll
