@@ -242,15 +242,14 @@ __device__ void analyse_gpu_priority(const GpParams &g, i64 t, GpSmem<LPT * S> &
     __syncwarp(gmask);
   }
   if (!dense) {  // any priorities: count the tasks that come before
+    i64 mine[S];
 #pragma unroll
-    for (int s = 0; s < S; ++s) {
-      const int i = lane + LPT * s;
-      int r = 0;
-      if (valid[s]) {
-        const i64 pi = sm.key[i];
-        for (int q = 0; q < n; ++q) r += (sm.key[q] > pi || (sm.key[q] == pi && q < i)) ? 1 : 0;
-      }
-      me.cpu_rank[s] = r;
+    for (int s = 0; s < S; ++s) mine[s] = valid[s] ? sm.key[lane + LPT * s] : 0, me.cpu_rank[s] = 0;
+    for (int q = 0; q < n; ++q) {
+      const i64 kq = sm.key[q];
+#pragma unroll
+      for (int s = 0; s < S; ++s)
+        me.cpu_rank[s] += (valid[s] && (kq > mine[s] || (kq == mine[s] && q < lane + LPT * s))) ? 1 : 0;
     }
   }
   __syncwarp(gmask);
@@ -293,24 +292,28 @@ __device__ void analyse_gpu_priority(const GpParams &g, i64 t, GpSmem<LPT * S> &
       if (valid[s]) sm.key[lane + LPT * s] = g.gpu_prio_in[a + lane + LPT * s];
     __syncwarp(gmask);
     int gpu_rank[S];
+    {
+      i64 mine[S];
 #pragma unroll
-    for (int s = 0; s < S; ++s) {
-      const int i = lane + LPT * s;
-      int r = 0;
-      if (valid[s]) {
-        const i64 pi = sm.key[i];
-        for (int q = 0; q < n; ++q) r += (sm.key[q] > pi || (sm.key[q] == pi && q < i)) ? 1 : 0;
-        sm.gpu_rank[i] = (short)r;
+      for (int s = 0; s < S; ++s) mine[s] = valid[s] ? sm.key[lane + LPT * s] : 0, gpu_rank[s] = 0;
+      for (int q = 0; q < n; ++q) {
+        const i64 kq = sm.key[q];
+#pragma unroll
+        for (int s = 0; s < S; ++s)
+          gpu_rank[s] += (valid[s] && (kq > mine[s] || (kq == mine[s] && q < lane + LPT * s))) ? 1 : 0;
       }
-      gpu_rank[s] = r;
+#pragma unroll
+      for (int s = 0; s < S; ++s)
+        if (valid[s]) sm.gpu_rank[lane + LPT * s] = (short)gpu_rank[s];
     }
     __syncwarp(gmask);
     int broken = 0;  // same core: the GPU order must equal the CPU order (Sec. 5.3)
+    for (int q = 0; q < n; ++q) {
+      const int core_q = sm.core[q], crank_q = sm.cpu_rank[q], grank_q = sm.gpu_rank[q];
 #pragma unroll
-    for (int s = 0; s < S; ++s)
-      if (valid[s])
-        for (int q = 0; q < n; ++q)
-          if (sm.core[q] == core[s] && sm.cpu_rank[q] < me.cpu_rank[s] && sm.gpu_rank[q] > gpu_rank[s]) broken = 1;
+      for (int s = 0; s < S; ++s)
+        if (valid[s] && core_q == core[s] && crank_q < me.cpu_rank[s] && grank_q > gpu_rank[s]) broken = 1;
+    }
     if (group_or<LPT>(broken, gmask)) {
 #pragma unroll
       for (int s = 0; s < S; ++s)
@@ -343,13 +346,18 @@ __device__ void analyse_gpu_priority(const GpParams &g, i64 t, GpSmem<LPT * S> &
       }
     }
     __syncwarp(gmask);
+    {  // the lowest CPU priority of every core starts as a candidate
+      bool lowest[S];
 #pragma unroll
-    for (int s = 0; s < S; ++s) {  // the lowest CPU priority of every core starts as a candidate
-      if (valid[s]) {
-        bool lowest = true;
-        for (int q = 0; q < n; ++q) lowest &= !(sm.core[q] == core[s] && sm.cpu_rank[q] > me.cpu_rank[s]);
-        if (lowest) atomicOr(&sm.cand[me.cpu_rank[s] >> 5], 1u << (me.cpu_rank[s] & 31));
+      for (int s = 0; s < S; ++s) lowest[s] = valid[s];
+      for (int q = 0; q < n; ++q) {
+        const int core_q = sm.core[q], rank_q = sm.cpu_rank[q];
+#pragma unroll
+        for (int s = 0; s < S; ++s) lowest[s] &= !(core_q == core[s] && rank_q > me.cpu_rank[s]);
       }
+#pragma unroll
+      for (int s = 0; s < S; ++s)
+        if (lowest[s]) atomicOr(&sm.cand[me.cpu_rank[s] >> 5], 1u << (me.cpu_rank[s] & 31));
     }
     __syncwarp(gmask);
     for (int level = 1; level <= n && sched == GCAPS_SCHED_YES; ++level) {
