@@ -94,6 +94,26 @@ def test_zero_overhead_and_literal_on_workloads():
         assert_parity(b, policy, 1000, 200, "sweep ovh=200")
 
 
+def test_priorities_that_are_not_a_dense_numbering():
+    """Sparse, tied and negative priority values on tasksets of every size bin: the kernels then
+    count the tasks that come before instead of subtracting from the largest priority."""
+    for name, count in (("sweep", 1500), ("large", 400), ("divergence", 2500)):
+        w = taskgen.WORKLOADS[name]
+        base = w.generate(29, count)
+        for what, f in (("sparse", lambda p: p * 3 + 5), ("tied", lambda p: p // 2),
+                        ("negative", lambda p: p * 7 - 1000)):
+            b = base.select(np.arange(base.n_tasksets))
+            b.priority = f(base.priority)
+            for policy in (0, 1, BUSY, 1 | BUSY):
+                assert_parity(b, policy, w.timeslice_us, w.overhead_us, "%s %s" % (name, what))
+            ts = binding.DeviceTasksets.from_host(b)
+            got = binding.rta_gpu_priority(ts, binding.ASSIGN, w.overhead_us)
+            torch.cuda.synchronize()
+            ref = rta.analyse_gpu_priority(b, rta.FLAG_ASSIGN, w.overhead_us)
+            for x, y in zip(got, ref):
+                assert np.array_equal(x.cpu().numpy(), y), "%s %s search" % (name, what)
+
+
 def test_size_bins_and_edges():
     """Sizes around every bin boundary, empty tasksets, the maximum size, in one batch."""
     rng = np.random.default_rng(5)
