@@ -170,3 +170,44 @@ int des_simulate(int n, const int64_t *T, const int64_t *prio, const int64_t *co
   return des_simulate_gp(n, T, prio, prio, core, offset, cseg_off, cseg, gseg_off, gm, ge, policy,
                          busy, L, horizon, max_resp, unfinished);
 }
+
+/*
+ * Brute force over release offsets: simulates the taskset once for EVERY offset vector
+ * (o_0, ..., o_{n-1}) with o_i in {0, step, 2*step, ...} below T_i, each run over two
+ * hyperperiods past the largest offset (hyper = lcm of the periods, passed in), and returns per
+ * task the largest response time seen in any run, a job still unfinished at a horizon counting
+ * with its age.  n_runs receives the number of offset vectors tried.  Arguments otherwise as
+ * des_simulate_gp.  Returns 0, or -1 if a run does not fit the simulator's limits.
+ */
+int des_sweep_offsets(int n, const int64_t *T, const int64_t *prio, const int64_t *gpu_prio,
+                      const int64_t *core, const int64_t *cseg_off, const int64_t *cseg,
+                      const int64_t *gseg_off, const int64_t *gm, const int64_t *ge, int policy,
+                      int busy, int64_t L, int64_t step, int64_t hyper, int64_t *worst,
+                      int64_t *n_runs) {
+  if (n < 1 || n > SIM_MAX_TASKS || step < 1) return -1;
+  int64_t off[SIM_MAX_TASKS], resp[SIM_MAX_TASKS], unfinished[SIM_MAX_TASKS];
+  for (int i = 0; i < n; ++i) off[i] = 0, worst[i] = 0;
+  *n_runs = 0;
+  for (;;) {
+    int64_t max_off = 0;
+    for (int i = 0; i < n; ++i)
+      if (off[i] > max_off) max_off = off[i];
+    if (des_simulate_gp(n, T, prio, gpu_prio, core, off, cseg_off, cseg, gseg_off, gm, ge, policy,
+                        busy, L, 2 * hyper + max_off + 1, resp, unfinished) != 0)
+      return -1;
+    *n_runs += 1;
+    for (int i = 0; i < n; ++i) {
+      if (resp[i] > worst[i]) worst[i] = resp[i];
+      if (unfinished[i] > worst[i]) worst[i] = unfinished[i];
+    }
+    int i = 0; /* next offset vector, first task fastest */
+    while (i < n) {
+      off[i] += step;
+      if (off[i] < T[i]) break;
+      off[i] = 0;
+      i += 1;
+    }
+    if (i == n) break;
+  }
+  return 0;
+}

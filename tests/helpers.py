@@ -14,15 +14,23 @@ BUSY, LITERAL, BEST_EFFORT = 0x100, 0x200, 0x800
 ALL_MODES = [0, BUSY, LITERAL, BUSY | LITERAL, 1, 1 | BUSY, 1 | LITERAL, 1 | BUSY | LITERAL]
 
 
-def parse_vectors(name):
-    """Reads a `task ... / case ...` fixture; returns (list of task dicts, list of cases)."""
-    tasks, cases = [], []
+def parse_vector_sets(name):
+    """Reads a fixture of `taskset <name>` / `task ...` / `case ...` lines; returns a list of
+    (taskset name, list of task dicts, list of cases), one entry per taskset of the file (a file
+    without `taskset` lines holds one unnamed taskset)."""
+    sets = []
     with open(os.path.join(GOLDEN, name)) as fh:
         for line in fh:
             line = line.split("#", 1)[0].strip()
             if not line:
                 continue
             tok = line.split()
+            if tok[0] == "taskset":
+                sets.append((tok[1], [], []))
+                continue
+            if not sets:
+                sets.append(("", [], []))
+            _, tasks, cases = sets[-1]
             kv = dict(x.split("=", 1) for x in tok[2:])
             if tok[0] == "task":
                 cseg = [int(x) for x in kv["cseg"].split(",") if x]
@@ -35,7 +43,14 @@ def parse_vectors(name):
                     BEST_EFFORT if kv.get("be", "0") == "1" else 0)
                 cases.append(dict(name=tok[1], policy=flags, L=int(kv["L"]), ovh=int(kv["ovh"]),
                                   expect=[int(x) for x in kv["expect"].split(",")]))
-    return tasks, cases
+    return sets
+
+
+def parse_vectors(name):
+    """Reads a one-taskset fixture; returns (list of task dicts, list of cases)."""
+    sets = parse_vector_sets(name)
+    assert len(sets) == 1, name
+    return sets[0][1], sets[0][2]
 
 
 def random_tasksets(rng, count, max_tasks=6, max_cores=3, periods=(20, 30, 40, 60, 80, 120, 200),

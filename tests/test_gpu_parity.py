@@ -11,7 +11,7 @@ import pytest
 
 from oracle import rta
 from paper_2406_05221_b200 import binding, taskgen
-from tests.helpers import ALL_MODES, BUSY, LITERAL, batch_of, parse_vectors, random_tasksets
+from tests.helpers import ALL_MODES, BUSY, LITERAL, batch_of, parse_vector_sets, random_tasksets
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -46,13 +46,15 @@ def assert_parity(batch, policy, L=1024, ovh=0, what=""):
     return w, s
 
 
-@pytest.mark.parametrize("fixture", ["table2_vectors.txt", "indirect_delay_vectors.txt"])
+@pytest.mark.parametrize("fixture", ["table2_vectors.txt", "indirect_delay_vectors.txt",
+                                     "same_core_jitter_vectors.txt"])
 def test_hand_derived_vectors(fixture):
-    tasks, cases = parse_vectors(fixture)
-    b = batch_of([tasks])
-    for c in cases:
-        w, s = gpu_run(b, c["policy"], c["L"], c["ovh"])
-        assert w.tolist() == c["expect"], c["name"]
+    for set_name, tasks, cases in parse_vector_sets(fixture):
+        b = batch_of([tasks])
+        for c in cases:
+            w, s = gpu_run(b, c["policy"], c["L"], c["ovh"])
+            assert w.tolist() == c["expect"], (set_name, c["name"])
+            assert s[0] == (1 if min(c["expect"]) >= 0 else 0), (set_name, c["name"])
 
 
 @pytest.mark.parametrize("policy", ALL_MODES)

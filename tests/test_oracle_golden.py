@@ -5,18 +5,21 @@ import numpy as np
 import pytest
 
 from oracle import rta, sim
-from tests.helpers import GOLDEN, batch_of, parse_vectors
+from tests.helpers import GOLDEN, batch_of, parse_vector_sets, parse_vectors
 
 
-@pytest.mark.parametrize("fixture", ["table2_vectors.txt", "indirect_delay_vectors.txt"])
+@pytest.mark.parametrize("fixture", ["table2_vectors.txt", "indirect_delay_vectors.txt",
+                                     "same_core_jitter_vectors.txt"])
 def test_hand_derived_vectors(fixture):
-    tasks, cases = parse_vectors(fixture)
-    assert cases
-    b = batch_of([tasks])
-    for c in cases:
-        wcrt, sched, _ = rta.analyse(b, c["policy"], c["L"], c["ovh"])
-        assert wcrt.tolist() == c["expect"], c["name"]
-        assert sched[0] == (1 if min(c["expect"]) >= 0 else 0), c["name"]
+    sets = parse_vector_sets(fixture)
+    assert sets
+    for set_name, tasks, cases in sets:
+        assert cases
+        b = batch_of([tasks])
+        for c in cases:
+            wcrt, sched, _ = rta.analyse(b, c["policy"], c["L"], c["ovh"])
+            assert wcrt.tolist() == c["expect"], (set_name, c["name"])
+            assert sched[0] == (1 if min(c["expect"]) >= 0 else 0), (set_name, c["name"])
 
 
 def test_table2_printed_verdict_and_schedule():
