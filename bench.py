@@ -29,17 +29,20 @@ if ROOT not in sys.path:
 METRIC = "tasksets analysed/sec (GCAPS & RR RTA)"
 UNIT = "tasksets/s"
 FALLBACK_HBM_GBS = 6650.0
-# plain-ALU peak of one B200: 148 SMs x 128 INT32 lanes x 1.965 GHz (integer lane-operations/s)
-ALU_PEAK_LANEOPS = 148 * 128 * 1.965e9
+# plain-ALU peak of one B200 from unit counts and clock, 148 SMs x 128 INT32 lanes x 1.965 GHz
+# (integer lane-operations/s): only the fallback when the issue-rate probe cannot run
+ALU_PEAK_DERIVED = 148 * 128 * 1.965e9
+# a workload larger than this is benchmarked one chunk at a time (the 10,000,000-taskset
+# workload is generated, analysed and verified in chunks of 1,000,000)
+MAX_TASKSETS_PER_GPU = 1_000_000
 K_TERM, K_SETUP = 6, 16   # algorithmic integer lane-operations per interference term / per task
 # kernels launched by one gcaps_rta_batch call: 3 plan kernels, one analysis kernel for the bins
 # of up to 32 tasks and one each for the 64-, 96-, 128-, 192- and 256-task bins
 LAUNCHES_PER_CALL = 9        # three plan kernels + one kernel per group of size bins
 LAUNCHES_PER_SMALL_CALL = 7  # batches of up to 8,192 tasksets: one plan kernel
-# DRAM bytes (read + write) per taskset of the analysis kernel on the 'large' workload, from the
-# ncu capture summarised in profiles/rta_kernel_large_131072_full.md (131,072 tasksets; traffic
-# grows in proportion to the tasksets of a launch).  Only reported while the kernel source is
-# the one the counters were taken from.
+# DRAM bytes (read + write) per taskset of the analysis kernel on the 'large' workload, from an
+# ncu capture of a 131,072-taskset launch (traffic grows in proportion to the tasksets of a
+# launch).  Only reported while the kernel source is the one the counters were taken from.
 CAPTURED_TRAFFIC = {
     "source_sha256": "992c86b02973be248905087f74519284979b90198204ab7a2bd867e3b67426d8",
     "workload": "large",
@@ -150,6 +153,37 @@ def oracle_sample(workload, first, count, budget_s, chunk=50_000, stream=0):
     return {"tasksets": done, "seconds": spent, "terms": terms, "sweeps": sweeps, "started": started}
 
 
+def _oracle_shard(job):
+    """Worker of the all-core CPU baseline: generates its own shard and times the oracle on it."""
+    os.environ["OMP_NUM_THREADS"] = "1"   # the generator's OpenMP loop stays on this core
+    name, first, count, stream = job
+    from paper_2406_05221_b200 import taskgen
+    r = oracle_sample(taskgen.WORKLOADS[name], first, count, 1e9, chunk=count, stream=stream)
+    return r["tasksets"], r["seconds"]
+
+
+def oracle_all_cores(workload, first, per_core, stream=0):
+    """The single-threaded oracle over disjoint shards of the workload, one per host core, in
+    processes started with `spawn` (a forked child of a process that has used CUDA hangs)."""
+    import multiprocessing as mp
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count() or 1
+    cores = max(1, min(cores, 256))
+    jobs = [(workload.name, first + k * per_core, per_core, stream) for k in range(cores)]
+    t0 = time.perf_counter()
+    with mp.get_context("spawn").Pool(cores) as pool:
+        got = pool.map(_oracle_shard, jobs, chunksize=1)
+    wall = time.perf_counter() - t0
+    tasksets = sum(g[0] for g in got)
+    slowest = max(g[1] for g in got)
+    return {"value": tasksets / slowest, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d tasksets per core on %d cores (disjoint shards), both policies; rate = all "
+                      "tasksets / the slowest core's oracle time (%.1f s); generation and process "
+                      "start excluded (%.1f s wall in all)" % (per_core, cores, slowest, wall)}
+
+
 def run_reference(args, workload):
     """The reference arm: the CPU oracle, single-threaded, on a bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -205,6 +239,12 @@ def main():
                     help="replay each call from a CUDA graph instead of enqueueing its launches again")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cpu-all-cores", action="store_true",
+                    help="skip the all-host-cores leg of the CPU baseline")
+    ap.add_argument("--cpu-all-cores-budget", type=float, default=6.0,
+                    help="seconds of oracle time per core for the all-cores leg")
+    ap.add_argument("--no-diagnostic", action="store_true",
+                    help="skip the secondary timing on tasksets that converge")
     args = ap.parse_args()
 
     from paper_2406_05221_b200 import taskgen
@@ -229,7 +269,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     binding.load_library()
 
-    per_gpu = args.tasksets or workload.n_tasksets
+    per_gpu = args.tasksets or min(workload.n_tasksets, MAX_TASKSETS_PER_GPU)
     first, count = sharding.weak_shard(rank, per_gpu)
     pinned = []
 
@@ -378,6 +418,43 @@ def main():
     if args.mode == "sweep":  # taskset analyses per second of the fused call alone
         value = world * count * len(pairs) / (per_policy_ms[0] * 1e-3)
 
+    # ---- beside the headline: the busy-waiting analyses, planning on its own, the integer peak --
+    def mean_ms(fn, n):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        e1.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    side = {}
+    if args.mode == "policies" and not fused and not args.graph:
+        n_side = max(3, min(args.steps, 20))
+        busy_ms = {nm: mean_ms(lambda pol=pol: binding.rta_batch(
+            ts, pol | binding.BUSY, L, ovh, out_wcrt=out_wcrt, out_sched=out_sched,
+            workspace=workspace, stream=stream), n_side) for nm, pol in zip(names, policies)}
+        plan_ms = mean_ms(lambda: binding.rta_plan(ts, workspace, stream=stream), n_side)
+        side["busy_waiting"] = {
+            "ms_per_launch": busy_ms, "value": count / (sum(busy_ms.values()) * 1e-3), "unit": UNIT,
+            "note": "the same batch under the busy-waiting lemmas (GCAPS_RTA_BUSY), %d steps, this rank" % n_side}
+        side["plan"] = {
+            "ms_per_call": plan_ms,
+            "share_of_call": {nm: plan_ms / ms for nm, ms in zip(names, per_policy_ms)},
+            "analysis_only_ms": {nm: ms - plan_ms for nm, ms in zip(names, per_policy_ms)},
+            "analysis_only_value": count / (sum(ms - plan_ms for ms in per_policy_ms) * 1e-3),
+            "note": "size binning of the batch (gcaps_rta_plan_batch) timed alone; `value` is plan + analysis"}
+    alu_peaks, alu_peak, alu_kind = None, ALU_PEAK_DERIVED, "derived (148 SMs x 128 lanes x 1.965 GHz)"
+    if rank == 0:
+        try:
+            alu_peaks = {nm: binding.int_issue_rate(kind, device=dev)
+                         for kind, nm in enumerate(("multiply_add", "add", "multiply_add_and_add"))}
+            alu_peak, alu_kind = alu_peaks["multiply_add_and_add"], "measured"
+        except Exception as exc:   # keep the derived figure, say why
+            alu_kind += "; probe failed: %s" % exc
+
     # ---- end to end through the host-buffer entry point (copies inside the timed region) -----
     e2e = None
     if not args.no_e2e:
@@ -425,23 +502,71 @@ def main():
                 "best_ms_per_launch": dict(zip(names, best_policy_ms)),
                 "frac_per_policy": {nm: bytes_per_call / (ms * 1e-3) / 1e9 / peak
                                     for nm, ms in zip(names, per_policy_ms)}}
+        roof["alu_peak_kind"] = alu_kind
+        roof["alu_peak_tlaneops"] = alu_peak / 1e12
+        roof["int_issue_probe_tlaneops"] = ({k: v / 1e12 for k, v in alu_peaks.items()}
+                                            if alu_peaks else None)
         if world == 1 and not args.no_cpu_baseline and args.mode == "policies":
             r = oracle_sample(workload, first, count, args.cpu_budget, stream=args.stream)
+            n_tasks_per_set = ts.n_tasks / max(1, ts.n_tasksets)
             cpu = {"value": r["tasksets"] / r["seconds"], "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": "first %d tasksets of the workload, both policies, %.1f s, generation excluded"
                              % (r["tasksets"], r["seconds"]),
-                   "terms_per_taskset": {"gcaps": r["terms"][0] / r["tasksets"], "rr": r["terms"][1] / r["tasksets"]}}
+                   "terms_per_taskset": {"gcaps": r["terms"][0] / r["tasksets"], "rr": r["terms"][1] / r["tasksets"]},
+                   "sweeps_per_taskset": {"gcaps": r["sweeps"][0] / r["tasksets"], "rr": r["sweeps"][1] / r["tasksets"]},
+                   # share of the tasks whose recurrence is started at all (the rest sit behind the
+                   # first deadline miss of their taskset)
+                   "tasks_analysed_fraction": {
+                       "gcaps": r["started"][0] / (r["tasksets"] * n_tasks_per_set),
+                       "rr": r["started"][1] / (r["tasksets"] * n_tasks_per_set)}}
+            if not args.no_cpu_all_cores:
+                per_core = max(200, min(int(cpu["value"] * args.cpu_all_cores_budget), count // 2))
+                cpu["all_cores"] = oracle_all_cores(workload, first, per_core, stream=args.stream)
             # which roofline binds: algorithmic integer work against algorithmic bytes
-            n_tasks_per_set = ts.n_tasks / max(1, ts.n_tasksets)
             t_mem = bytes_per_call / (peak * 1e9)
             terms = sum(r["terms"]) if fused else r["terms"][policies[dom]]
-            t_alu = count * (K_TERM * terms / r["tasksets"] + K_SETUP * n_tasks_per_set) / ALU_PEAK_LANEOPS
+            t_alu = count * (K_TERM * terms / r["tasksets"] + K_SETUP * n_tasks_per_set) / alu_peak
             roof["model_ms"] = {"hbm": 1e3 * t_mem, "alu": 1e3 * t_alu}
+            roof["frac_alu"] = t_alu / (per_policy_ms[dom] * 1e-3)
             if t_alu > t_mem:
-                ops = t_alu * ALU_PEAK_LANEOPS
+                ops = t_alu * alu_peak
                 ach = ops / (per_policy_ms[dom] * 1e-3)
-                roof.update(bound="alu", achieved=ach / 1e12, peak=ALU_PEAK_LANEOPS / 1e12,
-                            unit="Tlaneop/s", frac=ach / ALU_PEAK_LANEOPS)
+                roof.update(bound="alu", achieved=ach / 1e12, peak=alu_peak / 1e12,
+                            unit="Tlaneop/s", frac=ach / alu_peak)
+    # ---- a diagnostic beside the workload (never instead of it): tasksets of the same shape that
+    # converge, so that the recurrence of Eq. 1 runs for every task instead of ending at an early miss
+    diagnostic = None
+    if (rank == 0 and world == 1 and args.mode == "policies" and not fused and not args.graph
+            and workload.name == "large" and not args.no_diagnostic and not args.on_device_inputs):
+        from oracle import rta
+        light = taskgen.WORKLOADS["large_light"]
+        d_count = min(light.n_tasksets, 200_000)
+        d_batch = light.generate(0, d_count)
+        d_ts = binding.DeviceTasksets.from_host(d_batch, dev)
+        d_w = torch.empty(d_ts.n_tasks, dtype=torch.int64, device=dev)
+        d_s = torch.empty(d_ts.n_tasksets, dtype=torch.uint8, device=dev)
+        d_bytes = d_batch.input_bytes() + d_batch.output_bytes()
+        d_ms, d_sched, d_terms = {}, {}, {}
+        sample = d_batch.slice(0, 2000)
+        for nm, pol in zip(names, policies):
+            d_ms[nm] = mean_ms(lambda pol=pol: binding.rta_batch(
+                d_ts, pol, light.timeslice_us, light.overhead_us, out_wcrt=d_w, out_sched=d_s,
+                workspace=workspace, stream=stream), 20)
+            d_sched[nm] = float((d_s == 1).float().mean().item())
+            _, _, c = rta.analyse(sample, pol, light.timeslice_us, light.overhead_us)
+            d_terms[nm] = c.terms / 2000.0
+        diagnostic = {
+            "workload": light.name, "note": light.note, "tasksets": d_count,
+            "ms_per_launch": d_ms, "schedulable_fraction": d_sched,
+            "oracle_terms_per_taskset": d_terms,
+            "tasksets_per_s": {nm: d_count / (ms * 1e-3) for nm, ms in d_ms.items()},
+            "frac_hbm": {nm: d_bytes / (ms * 1e-3) / 1e9 / peak for nm, ms in d_ms.items()},
+            "frac_alu": {nm: d_count * (K_TERM * d_terms[nm] + K_SETUP * 80) / alu_peak / (ms * 1e-3)
+                         for nm, ms in d_ms.items()},
+            "alu_model": "%d lane-ops per interference term the oracle counts + %d per task, against "
+                         "the integer issue rate (%s)" % (K_TERM, K_SETUP, alu_kind)}
+        del d_ts, d_w, d_s
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -464,6 +589,9 @@ def main():
                             * (LAUNCHES_PER_SMALL_CALL if count <= 8192 else LAUNCHES_PER_CALL),
             "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
         }
+        line.update(side)
+        if diagnostic is not None:
+            line["recurrence_diagnostic"] = diagnostic
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -10,6 +10,17 @@
  *
  * All times are integer microseconds held as int64_t.  Nothing in this header is a torch type;
  * device buffers are plain device pointers owned by the caller.
+ *
+ * Host threads.  Every entry point may be called from several host threads at once.  The calls
+ * that work on device buffers keep no state between calls apart from per-device constants that
+ * are looked up once under a lock; concurrent calls must use different workspaces (and, to
+ * overlap on the GPU, different streams).  The host-buffer calls (gcaps_rta_batch_host,
+ * gcaps_rta_batch_host_multi, gcaps_rta_release_host) share one set of staging buffers and are
+ * serialised by a lock: a second thread waits until the first one's call has returned.
+ *
+ * Stream order.  The work of a call is complete, for everything enqueued on the same stream
+ * afterwards, when the stream reaches that later work: a copy of the results, a kernel reading
+ * them or the next call may follow without any host synchronisation.
  */
 #ifndef GCAPS_RTA_H_
 #define GCAPS_RTA_H_
@@ -163,7 +174,10 @@ size_t gcaps_rta_workspace_bytes(int64_t n_tasksets);
  * copies the inputs to the device in chunks of whole tasksets, runs gcaps_rta_batch on each
  * chunk, copies the results back and returns after everything has completed.  Device staging
  * memory is allocated on first use, grown on demand and kept until gcaps_rta_release_host();
- * page-locked host buffers give the best transfer rate but are not required.
+ * page-locked host buffers give the best transfer rate but are not required.  On an error return
+ * nothing of the call is still in flight: the caller's arrays may be freed at once (results of
+ * chunks that had completed may have been written).  One host-buffer call runs at a time per
+ * process; calls from other threads wait.
  */
 int gcaps_rta_batch_host(const gcaps_tasksets_t *ts, int64_t n_tasksets, int policy,
                          int64_t timeslice_us, int64_t ctx_switch_overhead_us, int64_t *out_wcrt,
@@ -287,7 +301,9 @@ int gcaps_rta_multi_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, int an
  *     GCAPS_ERR_TOO_LARGE and nothing is enqueued (split the batch, or use gcaps_rta_batch);
  *   - the call allocates nothing and frees nothing, on the host or on the device;
  *   - the first call on each device looks up the device address of the array (one cheap runtime
- *     query with that device current).  Make that first call outside any stream capture;
+ *     query with that device current).  Make that first call outside any stream capture.  The
+ *     address is kept for the life of the process and does not survive a cudaDeviceReset of that
+ *     device: do not call this entry point again after one;
  *   - every call on a device shares the one array and finds the previous call's plan in it.
  *     The kernels rewrite every word of it that they later read, so stale contents are harmless,
  *     but two calls whose kernels overlap on the GPU (different streams, or different host
@@ -357,6 +373,28 @@ int gcaps_gen_count(const gcaps_gen_params_t *params, int64_t first, int64_t cou
 int gcaps_gen_fill(const gcaps_gen_params_t *params, int64_t first, int64_t count,
                    const gcaps_tasksets_t *ts, void *workspace, size_t workspace_bytes,
                    void *stream);
+
+/*
+ * Measurement aids (not steps of the analysis; the paper reports no timing of its analysis at
+ * all, so it has no counterpart for either).
+ *
+ * gcaps_rta_plan_batch -- enqueues only the planning step of gcaps_rta_batch for this batch (the
+ * size-binned permutation of taskset indices in `workspace`), so that the cost of planning can
+ * be timed apart from the analysis.  Arguments and return codes as for gcaps_rta_batch.
+ *
+ * gcaps_rta_int_issue_probe -- enqueues one launch of a register-only integer kernel that fills
+ * every SM with independent arithmetic chains (8 per thread, 64 warps per SM) and reports how
+ * many 32-bit integer lane-operations the launch executes; divided by the launch's duration
+ * (CUDA events around the call) that is the device's integer issue rate, the bound beside HBM
+ * bandwidth for the recurrence of Eq. 1.  kind 0: multiply-add chains; 1: add chains; 2: one
+ * multiply-add and one add per step.  trips: 1 .. 2^24 loop trips of 16 chain steps each.
+ * scratch: DEVICE, one uint32 (never written in practice).  out_lane_ops: HOST, receives the
+ * count.  Asynchronous on `stream`.
+ */
+int gcaps_rta_plan_batch(const gcaps_tasksets_t *ts, int64_t n_tasksets, void *workspace,
+                         size_t workspace_bytes, void *stream);
+int gcaps_rta_int_issue_probe(int kind, int64_t trips, uint32_t *scratch, int64_t *out_lane_ops,
+                              void *stream);
 
 /* Frees the staging memory gcaps_rta_batch_host keeps on the current device. */
 void gcaps_rta_release_host(void);

@@ -6,6 +6,7 @@ missing or no B200 is present the calls raise.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 from typing import Dict, Optional, Tuple
@@ -39,7 +40,8 @@ EXPORTS = ("gcaps_rta_batch", "gcaps_rta_workspace_bytes", "gcaps_rta_batch_host
            "gcaps_rta_release_host", "gcaps_rta_validate", "gcaps_rta_strerror",
            "gcaps_rta_last_cuda_error", "gcaps_rta_version", "gcaps_rta_batch_static",
            "gcaps_rta_batch_host_multi", "gcaps_rta_gpu_priority_batch", "gcaps_rta_sweep_batch", "gcaps_rta_multi_batch",
-           "gcaps_gen_workspace_bytes", "gcaps_gen_count", "gcaps_gen_fill")
+           "gcaps_gen_workspace_bytes", "gcaps_gen_count", "gcaps_gen_fill",
+           "gcaps_rta_plan_batch", "gcaps_rta_int_issue_probe")
 
 _p64 = ctypes.POINTER(ctypes.c_int64)
 
@@ -110,6 +112,12 @@ def load_library(path: Optional[str] = None):
                                        ctypes.POINTER(CTasksets), ctypes.c_void_p, ctypes.c_size_t,
                                        ctypes.c_void_p]
         lib.gcaps_gen_fill.restype = ctypes.c_int
+        lib.gcaps_rta_plan_batch.argtypes = [ctypes.POINTER(CTasksets), ctypes.c_int64, ctypes.c_void_p,
+                                             ctypes.c_size_t, ctypes.c_void_p]
+        lib.gcaps_rta_plan_batch.restype = ctypes.c_int
+        lib.gcaps_rta_int_issue_probe.argtypes = [ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, _p64,
+                                                  ctypes.c_void_p]
+        lib.gcaps_rta_int_issue_probe.restype = ctypes.c_int
         lib.gcaps_rta_release_host.argtypes = []
         lib.gcaps_rta_release_host.restype = None
         lib.gcaps_rta_validate.argtypes = [ctypes.POINTER(CTasksets), ctypes.c_int64,
@@ -121,6 +129,19 @@ def load_library(path: Optional[str] = None):
         lib.gcaps_rta_version.restype = ctypes.c_int
         _lib = lib
     return _lib
+
+
+@contextlib.contextmanager
+def _device_and_stream(dev, stream):
+    """Makes ``dev`` the current device and ``stream`` (default: torch's current one) the current
+    stream.  Tensors the wrappers create inside (outputs, workspace) then belong to the stream the
+    kernels run on, so torch's allocator cannot hand their memory to someone else while those
+    kernels are still in flight."""
+    import torch
+    with torch.cuda.device(dev):
+        st = stream if stream is not None else torch.cuda.current_stream(dev)
+        with torch.cuda.stream(st):
+            yield st
 
 
 def _check(rc: int):
@@ -165,7 +186,7 @@ def rta_batch(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, overhea
     import torch
     lib = load_library()
     dev = ts.t["task_off"].device
-    with torch.cuda.device(dev):
+    with _device_and_stream(dev, stream) as st:
         if out_wcrt is None:
             out_wcrt = torch.empty(ts.n_tasks, dtype=torch.int64, device=dev)
         if out_sched is None:
@@ -173,7 +194,6 @@ def rta_batch(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, overhea
         need = workspace_bytes(ts.n_tasksets)
         if workspace is None:
             workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
-        st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_batch(ctypes.byref(ts.c), ts.n_tasksets, policy, timeslice_us, overhead_us,
                                  out_wcrt.data_ptr(), out_sched.data_ptr(), workspace.data_ptr(),
                                  workspace.numel(), st.cuda_stream)
@@ -192,7 +212,7 @@ def rta_sweep(ts: DeviceTasksets, policy: int, timeslices_us, overheads_us, want
     k = len(overheads_us)
     Ls = (ctypes.c_int64 * k)(*[int(x) for x in timeslices_us]) if timeslices_us is not None else None
     ov = (ctypes.c_int64 * k)(*[int(x) for x in overheads_us])
-    with torch.cuda.device(dev):
+    with _device_and_stream(dev, stream) as st:
         if out_wcrt is None and want_wcrt:
             out_wcrt = torch.empty((k, ts.n_tasks), dtype=torch.int64, device=dev)
         if out_sched is None:
@@ -200,7 +220,6 @@ def rta_sweep(ts: DeviceTasksets, policy: int, timeslices_us, overheads_us, want
         need = workspace_bytes(ts.n_tasksets)
         if workspace is None:
             workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
-        st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_sweep_batch(ctypes.byref(ts.c), ts.n_tasksets, policy, k, Ls, ov,
                                        out_wcrt.data_ptr() if out_wcrt is not None else None,
                                        out_sched.data_ptr(), workspace.data_ptr(), workspace.numel(),
@@ -222,14 +241,13 @@ def rta_multi(ts: DeviceTasksets, analyses: int, timeslices_us=(1024,), overhead
     n_pts, k = len(overheads_us), bin(analyses & 15).count("1")
     Ls = (ctypes.c_int64 * n_pts)(*[int(x) for x in timeslices_us]) if timeslices_us is not None else None
     ov = (ctypes.c_int64 * n_pts)(*[int(x) for x in overheads_us])
-    with torch.cuda.device(dev):
+    with _device_and_stream(dev, stream) as st:
         if out_wcrt is None and want_wcrt:
             out_wcrt = torch.empty((n_pts, k, ts.n_tasks), dtype=torch.int64, device=dev)
         if out_sched is None:
             out_sched = torch.empty((n_pts, k, max(ts.n_tasksets, 0)), dtype=torch.uint8, device=dev)
         if workspace is None:
             workspace = torch.empty(max(workspace_bytes(ts.n_tasksets), 256), dtype=torch.uint8, device=dev)
-        st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_multi_batch(ctypes.byref(ts.c), ts.n_tasksets, analyses, flags, n_pts, Ls, ov,
                                        out_wcrt.data_ptr() if out_wcrt is not None else None,
                                        out_sched.data_ptr(), workspace.data_ptr(), workspace.numel(),
@@ -250,12 +268,11 @@ def rta_batch_static(ts: DeviceTasksets, policy: int, timeslice_us: int = 1024, 
     import torch
     lib = load_library()
     dev = ts.t["task_off"].device
-    with torch.cuda.device(dev):
+    with _device_and_stream(dev, stream) as st:
         if out_wcrt is None:
             out_wcrt = torch.empty(ts.n_tasks, dtype=torch.int64, device=dev)
         if out_sched is None:
             out_sched = torch.empty(max(ts.n_tasksets, 0), dtype=torch.uint8, device=dev)
-        st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_batch_static(ctypes.byref(ts.c), ts.n_tasksets, policy, timeslice_us,
                                         overhead_us, out_wcrt.data_ptr(), out_sched.data_ptr(),
                                         st.cuda_stream)
@@ -271,13 +288,12 @@ def rta_gpu_priority(ts: DeviceTasksets, flags: int = 0, overhead_us: int = 0, g
     import torch
     lib = load_library()
     dev = ts.t["task_off"].device
-    with torch.cuda.device(dev):
+    with _device_and_stream(dev, stream) as st:
         out_wcrt = torch.full((ts.n_tasks,), WCRT_INVALID, dtype=torch.int64, device=dev)
         out_sched = torch.full((max(ts.n_tasksets, 0),), SCHED_INVALID, dtype=torch.uint8, device=dev)
         out_gp = torch.zeros(ts.n_tasks, dtype=torch.int64, device=dev)
         if workspace is None:
             workspace = torch.empty(max(workspace_bytes(ts.n_tasksets), 256), dtype=torch.uint8, device=dev)
-        st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_gpu_priority_batch(
             ctypes.byref(ts.c), ts.n_tasksets, flags, overhead_us,
             gpu_priority.data_ptr() if gpu_priority is not None else None, out_gp.data_ptr(),
@@ -298,8 +314,7 @@ def generate_device(params: GenParams, first: int, count: int, device="cuda:0", 
     lib = load_library()
     dev = torch.device(device)
     cp = params.int_params()
-    with torch.cuda.device(dev):
-        st = stream if stream is not None else torch.cuda.current_stream(dev)
+    with _device_and_stream(dev, stream) as st:
         ws = torch.empty(max(int(lib.gcaps_gen_workspace_bytes(ctypes.byref(cp), count)), 256), dtype=torch.uint8,
                          device=dev)
         totals = torch.zeros(3, dtype=torch.int64, device=dev)
@@ -328,14 +343,48 @@ def generate_device(params: GenParams, first: int, count: int, device="cuda:0", 
     return ts
 
 
+def rta_plan(ts: DeviceTasksets, workspace, stream=None):
+    """gcaps_rta_plan_batch: only the planning step of a call (for timing it apart)."""
+    import torch
+    lib = load_library()
+    dev = ts.t["task_off"].device
+    with _device_and_stream(dev, stream) as st:
+        rc = lib.gcaps_rta_plan_batch(ctypes.byref(ts.c), ts.n_tasksets, workspace.data_ptr(),
+                                      workspace.numel(), st.cuda_stream)
+    _check(rc)
+
+
+def int_issue_rate(kind: int = 2, trips: int = 2048, repeats: int = 5, device="cuda:0") -> float:
+    """Integer lane-operations per second of the device, measured with gcaps_rta_int_issue_probe
+    (kind 0: multiply-add chains, 1: add chains, 2: both); best of ``repeats`` launches."""
+    import torch
+    lib = load_library()
+    dev = torch.device(device)
+    with torch.cuda.device(dev):
+        scratch = torch.zeros(1, dtype=torch.int32, device=dev)
+        st = torch.cuda.current_stream(dev)
+        ops = ctypes.c_int64(0)
+        best = None
+        for k in range(repeats + 1):   # the first launch is a warm-up
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            _check(lib.gcaps_rta_int_issue_probe(kind, trips, scratch.data_ptr(), ctypes.byref(ops),
+                                                 st.cuda_stream))
+            e1.record(st)
+            e1.synchronize()
+            ms = e0.elapsed_time(e1)
+            if k > 0 and (best is None or ms < best):
+                best = ms
+    return ops.value / (best * 1e-3)
+
+
 def rta_validate(ts: DeviceTasksets, stream=None):
     """gcaps_rta_validate: int32 error mask per taskset (CUDA tensor)."""
     import torch
     lib = load_library()
     dev = ts.t["task_off"].device
-    with torch.cuda.device(dev):
+    with _device_and_stream(dev, stream) as st:
         out = torch.empty(max(ts.n_tasksets, 0), dtype=torch.int32, device=dev)
-        st = stream if stream is not None else torch.cuda.current_stream(dev)
         rc = lib.gcaps_rta_validate(ctypes.byref(ts.c), ts.n_tasksets, out.data_ptr(), st.cuda_stream)
     _check(rc)
     return out

@@ -437,13 +437,13 @@ static_assert(kSmallWarpBytes % 16 == 0, "every warp's area starts 16-byte align
 // the four bins of up to 32 tasks: (lanes per taskset, tasks per lane) as in the default analysis
 __global__ void __launch_bounds__(kBlockThreads) gpu_priority_small_kernel(GpParams g) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
-  asm volatile("griddepcontrol.launch_dependents;");
+  let_dependents_start();  // the kernel of the next size bin shares no data with this one
   unsigned char *mine = smem_raw + (threadIdx.x >> 5) * kSmallWarpBytes;
   run_bin<16, 2>(g, 3, mine);
   run_bin<8, 3>(g, 2, mine);
   run_bin<8, 2>(g, 1, mine);
   run_bin<8, 1>(g, 0, mine);
+  wait_for_previous_grid();
 }
 
 // one bin of larger tasksets, a warp per taskset.  Five blocks per SM (96 registers): the search is
@@ -452,8 +452,9 @@ __global__ void __launch_bounds__(kBlockThreads) gpu_priority_small_kernel(GpPar
 template <int S>
 __global__ void __launch_bounds__(kBlockThreads, 5) gpu_priority_big_kernel(GpParams g, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  asm volatile("griddepcontrol.launch_dependents;");
+  let_dependents_start();
   run_bin<32, S>(g, bin, smem_raw + (threadIdx.x >> 5) * warp_bytes<32, S>());
+  wait_for_previous_grid();
 }
 
 template <int S>

@@ -33,6 +33,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "rta_common.cuh"
 
 using namespace gcaps_detail;
@@ -1137,26 +1139,26 @@ constexpr int kSmallWarpWords =
 template <int MODE>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(3)) rta_small_kernel(KParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
-  asm volatile("griddepcontrol.launch_dependents;");
+  let_dependents_start();  // the kernel of the next size bin shares no data with this one
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
   run_bin<16, 2, 1 << MODE>(p, 3, warp_buf, ahead);
   run_bin<8, 3, 1 << MODE>(p, 2, warp_buf, ahead);
   run_bin<8, 2, 1 << MODE>(p, 1, warp_buf, ahead);
   run_bin<8, 1, 1 << MODE>(p, 0, warp_buf, ahead);
+  wait_for_previous_grid();
 }
 
 // One bin of larger tasksets (a warp per taskset, 2, 3, 4, 6 or 8 tasks per lane) per launch.
 template <int SLOTS, int MODE>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kernel(KParams p, int bin) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
-  asm volatile("griddepcontrol.launch_dependents;");
+  let_dependents_start();  // the kernel of the next size bin shares no data with this one
   constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
   run_bin<32, SLOTS, 1 << MODE>(p, bin, warp_buf, ahead);
+  wait_for_previous_grid();
 }
 
 // The same launches for a fused sweep: every taskset is read once and analysed under all the
@@ -1165,26 +1167,26 @@ template <int MASK>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(3))
 rta_small_sweep_kernel(KParams p, const __grid_constant__ SweepArgs sw) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
-  asm volatile("griddepcontrol.launch_dependents;");
+  let_dependents_start();  // the kernel of the next size bin shares no data with this one
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kSmallWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kSmallWarpWords - kAheadWords);
   run_bin<16, 2, MASK, true>(p, 3, warp_buf, ahead, &sw);
   run_bin<8, 3, MASK, true>(p, 2, warp_buf, ahead, &sw);
   run_bin<8, 2, MASK, true>(p, 1, warp_buf, ahead, &sw);
   run_bin<8, 1, MASK, true>(p, 0, warp_buf, ahead, &sw);
+  wait_for_previous_grid();
 }
 
 template <int SLOTS, int MASK>
 __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS))
 rta_big_sweep_kernel(KParams p, int bin, const __grid_constant__ SweepArgs sw) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // the kernel of the next size bin may start as blocks of this one leave (it shares no data)
-  asm volatile("griddepcontrol.launch_dependents;");
+  let_dependents_start();  // the kernel of the next size bin shares no data with this one
   constexpr int kWarpWords = bin_warp_words<32, SLOTS>() + kAheadWords;
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
   run_bin<32, SLOTS, MASK, true>(p, bin, warp_buf, ahead, &sw);
+  wait_for_previous_grid();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1232,6 +1234,7 @@ size_t plan_blocks(int64_t n_tasksets) { return (size_t)((n_tasksets + kPlanItem
 namespace gcaps_detail {
 
 thread_local int g_last_cuda_error = 0;
+std::mutex g_init_mutex;
 
 static DeviceInfo g_dev[64];
 
@@ -1243,6 +1246,7 @@ int device_info(DeviceInfo *out) {
     return GCAPS_ERR_NO_DEVICE;
   }
   if (dev < 0 || dev >= 64) return GCAPS_ERR_NO_DEVICE;
+  std::lock_guard<std::mutex> lock(g_init_mutex);
   if (g_dev[dev].ok == 0) {
     int major = 0, sms = 0;
     e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
@@ -1442,6 +1446,19 @@ struct HostStage {
   bool streams_ok;
 };
 HostStage g_stage = {{nullptr, nullptr}, {0, 0}, {nullptr, nullptr}, -1, false};
+std::mutex g_stage_mutex;  // one host-buffer call at a time owns the staging slots
+
+void release_stage_locked() {
+  for (int k = 0; k < 2; ++k) {
+    if (g_stage.dev[k]) cudaFree(g_stage.dev[k]);
+    g_stage.dev[k] = nullptr;
+    g_stage.dev_bytes[k] = 0;
+    if (g_stage.streams_ok && g_stage.stream[k]) cudaStreamDestroy(g_stage.stream[k]);
+    g_stage.stream[k] = nullptr;
+  }
+  g_stage.streams_ok = false;
+  g_stage.device = -1;
+}
 
 // Workspace of gcaps_rta_batch_static: lives in the library image, one copy per device that
 // loads it.  In host code this name is only a handle for cudaGetSymbolAddress, never an address
@@ -1541,23 +1558,28 @@ int gcaps_rta_batch_static(const gcaps_tasksets_t *ts, int64_t n_tasksets, int p
     g_last_cuda_error = (int)e;
     return GCAPS_ERR_NO_DEVICE;
   }
-  if (!g_static_scratch_ptr[dev]) {
-    // once per device, with that device current: the array's address on this device
-    void *ptr = nullptr;
-    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
-    if (e != cudaSuccess || !ptr) {
-      g_last_cuda_error = (int)e;
-      return GCAPS_ERR_CUDA;
+  void *scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_init_mutex);
+    if (!g_static_scratch_ptr[dev]) {
+      // once per device, with that device current: the array's address on this device
+      void *ptr = nullptr;
+      e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+      if (e != cudaSuccess || !ptr) {
+        g_last_cuda_error = (int)e;
+        return GCAPS_ERR_CUDA;
+      }
+      g_static_scratch_ptr[dev] = ptr;
     }
-    g_static_scratch_ptr[dev] = ptr;
+    scratch = g_static_scratch_ptr[dev];
   }
   KParams p;
   fill_params(&p, ts, n_tasksets, policy, timeslice_us, ctx_switch_overhead_us, out_wcrt, out_sched);
   // Nothing in the array has to be cleared first: the plan kernels write the header (counts,
   // starts, zeroed work counters), every per-block count and every permutation entry that the
   // analysis kernels of this call read.
-  return enqueue_batch(p, g_static_scratch_ptr[dev], (size_t)GCAPS_RTA_STATIC_SCRATCH_BYTES,
-                       di.sm_count, (cudaStream_t)stream);
+  return enqueue_batch(p, scratch, (size_t)GCAPS_RTA_STATIC_SCRATCH_BYTES, di.sm_count,
+                       (cudaStream_t)stream);
 }
 
 int gcaps_rta_validate(const gcaps_tasksets_t *ts, int64_t n_tasksets, int32_t *out_err,
@@ -1590,15 +1612,8 @@ int gcaps_rta_validate(const gcaps_tasksets_t *ts, int64_t n_tasksets, int32_t *
   } while (0)
 
 void gcaps_rta_release_host(void) {
-  for (int k = 0; k < 2; ++k) {
-    if (g_stage.dev[k]) cudaFree(g_stage.dev[k]);
-    g_stage.dev[k] = nullptr;
-    g_stage.dev_bytes[k] = 0;
-    if (g_stage.streams_ok && g_stage.stream[k]) cudaStreamDestroy(g_stage.stream[k]);
-    g_stage.stream[k] = nullptr;
-  }
-  g_stage.streams_ok = false;
-  g_stage.device = -1;
+  std::lock_guard<std::mutex> lock(g_stage_mutex);
+  release_stage_locked();
 }
 
 constexpr int kMaxHostPolicies = GCAPS_RTA_MAX_HOST_POLICIES;
@@ -1680,6 +1695,17 @@ static int host_chunk(const gcaps_tasksets_t *ts, int64_t t, int64_t t1, const i
   return GCAPS_OK;
 }
 
+// An error in a later chunk: earlier chunks' copies into the caller's arrays may still be in
+// flight on the staging streams; nothing of this call may touch the caller's memory once it has
+// returned.  Keeps the CUDA error code the failing step recorded.
+static int drain_stage(int rc) {
+  const int keep = g_last_cuda_error;
+  for (int k = 0; k < 2; ++k)
+    if (g_stage.streams_ok && g_stage.stream[k]) cudaStreamSynchronize(g_stage.stream[k]);
+  g_last_cuda_error = keep;
+  return rc;
+}
+
 // True if the task range [k0, k1] is inside the arrays and both segment offset arrays are
 // non-decreasing and in range over it.
 static bool host_range_is_canonical(const gcaps_tasksets_t *ts, int64_t k0, int64_t k1) {
@@ -1715,10 +1741,11 @@ int gcaps_rta_batch_host_multi(const gcaps_tasksets_t *ts, int64_t n_tasksets, c
   DeviceInfo di;
   rc = device_info(&di);
   if (rc != GCAPS_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_stage_mutex);
   int dev = 0;
   HOST_TRY(cudaGetDevice(&dev));
   if (g_stage.device != dev) {
-    gcaps_rta_release_host();
+    release_stage_locked();
     g_stage.device = dev;
   }
   if (!g_stage.streams_ok) {
@@ -1744,7 +1771,7 @@ int gcaps_rta_batch_host_multi(const gcaps_tasksets_t *ts, int64_t n_tasksets, c
     if (t1 > t && host_range_is_canonical(ts, k0, k1)) {
       rc = host_chunk(ts, t, t1, policies, n_policies, timeslice_us, ctx_switch_overhead_us,
                       out_wcrt, out_sched, slot, di.sm_count);
-      if (rc != GCAPS_OK) return rc;
+      if (rc != GCAPS_OK) return drain_stage(rc);
       slot ^= 1;
       t = t1;
       continue;
@@ -1764,7 +1791,7 @@ int gcaps_rta_batch_host_multi(const gcaps_tasksets_t *ts, int64_t n_tasksets, c
       } else {
         rc = host_chunk(ts, t, t + 1, policies, n_policies, timeslice_us, ctx_switch_overhead_us,
                         out_wcrt, out_sched, slot, di.sm_count);
-        if (rc != GCAPS_OK) return rc;
+        if (rc != GCAPS_OK) return drain_stage(rc);
         slot ^= 1;
       }
     }

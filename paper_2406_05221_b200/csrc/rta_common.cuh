@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/gcaps_rta.h"
 
 namespace gcaps_detail {
@@ -147,12 +149,31 @@ __host__ __device__ __forceinline__ void make_reciprocal(u32 d, u32 &magic, u32 
 #endif
 }
 
+// The kernels of the size bins of one call follow one another in the caller's stream and share no
+// data.  Each lets its dependents go at entry, and all but the first are launched with
+// programmatic stream serialisation, so the next bin's blocks start as this one's leave.  A grid
+// launched that way could otherwise also COMPLETE before its predecessor, and whatever the stream
+// runs next (a copy of the results, the plan kernels of the next call rewriting the workspace)
+// would then overtake a kernel that is still writing.  So every kernel ends with
+// griddepcontrol.wait: no grid retires before the grid in front of it has completed and its writes
+// are visible, completion is transitive along the chain, and the first kernel of the chain is an
+// ordinary launch that waited for everything before it.
+__device__ __forceinline__ void let_dependents_start() {
+  asm volatile("griddepcontrol.launch_dependents;");
+}
+__device__ __forceinline__ void wait_for_previous_grid() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Launches `kernel` (a persistent kernel of kBlockThreads threads needing `smem` bytes) with as
 // many blocks as the device keeps resident, but never more than the batch could feed.
 // overlap_previous: the kernel launched just before on this stream works on other data (another
-// size bin) and has let its dependents go (griddepcontrol.launch_dependents), so this one is
-// launched with programmatic stream serialisation and fills the SMs as that one's blocks leave
-// instead of waiting for its last block.  It needs nothing that kernel writes.
+// size bin) and has let its dependents go (let_dependents_start), so this one is launched with
+// programmatic stream serialisation and fills the SMs as that one's blocks leave instead of
+// waiting for its last block.  It needs nothing that kernel writes, and it must end with
+// wait_for_previous_grid().
+extern std::mutex g_init_mutex;  // guards the once-per-device set-up steps of the library
+
 template <typename... Args>
 cudaError_t launch_persistent_ex(bool overlap_previous, void (*kernel)(Args...), int *blocks_per_sm,
                                  size_t smem, long long want, int sm_count, cudaStream_t st, Args... args) {
@@ -160,15 +181,18 @@ cudaError_t launch_persistent_ex(bool overlap_previous, void (*kernel)(Args...),
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   dev &= 63;
-  if (blocks_per_sm[dev] == 0) {  // first use on this device
+  int resident = __atomic_load_n(&blocks_per_sm[dev], __ATOMIC_ACQUIRE);
+  if (resident == 0) {  // first use on this device (host threads may get here together)
+    std::lock_guard<std::mutex> lock(g_init_mutex);
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 1;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlockThreads, smem);
     if (e != cudaSuccess) return e;
-    blocks_per_sm[dev] = per_sm < 1 ? 1 : per_sm;
+    resident = per_sm < 1 ? 1 : per_sm;
+    __atomic_store_n(&blocks_per_sm[dev], resident, __ATOMIC_RELEASE);
   }
-  long long grid = (long long)sm_count * blocks_per_sm[dev];
+  long long grid = (long long)sm_count * resident;
   if (grid > want) grid = want;
   if (grid < 1) grid = 1;
   if (!overlap_previous) {

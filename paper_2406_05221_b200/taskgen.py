@@ -370,6 +370,16 @@ def _workloads() -> Dict[str, Workload]:
                    period_us=(1e2, 1e7), harmonic_frac=0.5, gpu_mode=1, gpu_segments=(0, 8),
                    gpu_ratio=(0.05, 0.9))],
         note="10,000,000 tasksets, 2-16 cores x 2-12 tasks, 0-8 segments, half harmonic periods")
+    # a diagnostic beside the five benchmark workloads: the shape of `large` with so little load
+    # and overhead that (under GCAPS) every taskset converges, so that the recurrence runs for all
+    # 80 tasks of a taskset instead of stopping at an early deadline miss
+    w["large_light"] = Workload(
+        "large_light", 200_000,
+        [GenParams(seed=6, cores=(8, 8), tasks_per_core=(10, 10), util_per_core=(0.05, 0.2),
+                   period_us=(1e3, 1e6), gpu_frac=0.8, gpu_segments=(1, 5), gpu_ratio=(0.1, 0.3))],
+        overhead_us=5,
+        note="200,000 tasksets shaped like 'large' (8 cores x 10 tasks, 80% GPU tasks) with "
+             "U/core 0.05-0.2, GPU share 10-30%, overhead 5 us: schedulable under GCAPS")
     return w
 
 

@@ -75,3 +75,29 @@ def test_argument_errors_need_no_device(lib):
         assert rc == binding.ERR_INVALID_ARG, kw
     assert lib.gcaps_rta_batch(None, 0, 0, 1, 0, None, None, None, 0, None) == binding.ERR_INVALID_ARG
     assert lib.gcaps_rta_batch(ctypes.byref(c), 0, 0, 1, 0, None, None, None, 0, None) == binding.OK
+
+
+def test_host_only_calls_from_several_threads(lib):
+    """The entry points may be called from several host threads at once; what can be checked
+    without a device: argument errors and the pure host computations give the same answers."""
+    import threading
+    want = [binding.workspace_bytes(n) for n in range(0, 200_000, 997)]
+    c = binding.CTasksets()
+    wrong = []
+
+    def run():
+        for _ in range(20):
+            if [binding.workspace_bytes(n) for n in range(0, 200_000, 997)] != want:
+                wrong.append("workspace_bytes")
+            for call in (lambda: lib.gcaps_rta_batch(ctypes.byref(c), 1, 7, 1, 0, None, None, None, 0, None),
+                         lambda: lib.gcaps_rta_batch_host(ctypes.byref(c), 1, 0, 1, -1, None, None),
+                         lambda: lib.gcaps_rta_batch_static(ctypes.byref(c), 1, 1, 0, 0, None, None, None)):
+                if call() != binding.ERR_INVALID_ARG:
+                    wrong.append("argument error")
+
+    threads = [threading.Thread(target=run) for _ in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not wrong, wrong

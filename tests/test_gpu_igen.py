@@ -1,12 +1,15 @@
 """On-device taskset generation (gcaps_gen_count / gcaps_gen_fill) through the C-ABI: bit-exact
-against the host build of the same integer-only generator, and the analysis of tasksets that were
-generated on the device against the CPU oracle on their host-generated twins."""
+against the generator's oracle (oracle/igen_oracle.py, plain Python integers, no code in common
+with the library) on samples of every workload, against the host build of the library's own
+generator on larger ranges, and the analysis of tasksets that were generated on the device against
+the CPU oracle on their host-generated twins."""
 import ctypes
 
 import numpy as np
 import pytest
 
 from oracle import rta
+from oracle.igen_oracle import reference_taskset
 from paper_2406_05221_b200 import binding, taskgen
 
 torch = pytest.importorskip("torch")
@@ -25,6 +28,31 @@ def assert_same(ts, batch, what):
         got = ts.t[f].cpu().numpy()
         assert got.shape == getattr(batch, f).shape, (what, f)
         assert np.array_equal(got, getattr(batch, f)), (what, f)
+
+
+@pytest.mark.parametrize("name,stream,first,count", [
+    ("pr1", 0, 0, 300), ("sweep", 0, 77, 200), ("sweep", 4, 50_000, 200), ("sweep", 8, 99_900, 100),
+    ("large", 0, 999_950, 50), ("rr_model", 0, 123_456, 200), ("divergence", 0, 9_999_900, 100),
+    ("divergence", 0, 31, 150)])
+def test_device_generation_equals_the_generator_oracle(name, stream, first, count):
+    """The device output against the plain-integer oracle of the generator, taskset by taskset."""
+    w = taskgen.WORKLOADS[name]
+    ts = binding.generate_device(w.streams[stream], first, count)
+    torch.cuda.synchronize()
+    p = w.streams[stream].int_params()
+    want = taskgen.TasksetBatch.from_tasksets([reference_taskset(p, first + t) for t in range(count)])
+    assert_same(ts, want, "%s/%d against the oracle" % (name, stream))
+
+
+def test_device_generation_at_the_range_ends_equals_the_generator_oracle():
+    params = taskgen.GenParams(seed=42, cores=(1, 3), tasks_per_core=(1, 3), util_per_core=(0.5, 0.99),
+                               period_us=(1e6, 1.07e9), gpu_mode=1, gpu_segments=(0, 16),
+                               gpu_ratio=(0.0, 0.99), harmonic_frac=0.5, wfd=True)
+    ts = binding.generate_device(params, 3, 400)
+    torch.cuda.synchronize()
+    p = params.int_params()
+    want = taskgen.TasksetBatch.from_tasksets([reference_taskset(p, 3 + t) for t in range(400)])
+    assert_same(ts, want, "range ends against the oracle")
 
 
 @pytest.mark.parametrize("name,stream,first,count", [

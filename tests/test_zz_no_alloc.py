@@ -3,17 +3,17 @@
 Some users of the library run where cudaMalloc is not theirs to call (a plug-in whose host owns
 the allocator, a process that must not allocate after start-up).  For them the library carries
 its own fixed scratch array.  This test calls that entry point through the C-ABI twice in a row
-and requires exactly the outputs of the ordinary entry point (all values are integers, so the
-tolerance is zero), with the second call finding the first call's left-overs in the scratch.
-
-The file name sorts last on purpose: a run that stops at the first failure has then already run
-every other test.
+and requires exactly the outputs of the ordinary entry point and of the CPU oracle (all values
+are integers, so the tolerance is zero), with the second call finding the first call's
+left-overs in the scratch; it also checks that such a call leaves the amount of free device
+memory untouched.
 """
 import ctypes
 
 import numpy as np
 import pytest
 
+from oracle import rta
 from paper_2406_05221_b200 import binding, taskgen
 
 torch = pytest.importorskip("torch")
@@ -36,6 +36,10 @@ def _both(batch, policy, L, ovh):
     binding.rta_batch_static(ts, policy, L, ovh, out_wcrt=out_w, out_sched=out_s)
     torch.cuda.synchronize()
     assert torch.equal(out_w, ref_w) and torch.equal(out_s, ref_s)
+    # the oracle itself, not only the other entry point
+    w_cpu, s_cpu, _ = rta.analyse(batch, policy, L, ovh)
+    assert np.array_equal(out_w.cpu().numpy(), w_cpu)
+    assert np.array_equal(out_s.cpu().numpy(), s_cpu)
 
 
 def test_two_calls_in_a_row_match_the_workspace_entry_point():
@@ -67,3 +71,31 @@ def test_limit_is_enforced_without_enqueuing_anything():
     reps = binding.STATIC_MAX_TASKSETS // 1000 + 1
     at_limit = taskgen.TasksetBatch.concat([edge] * reps).slice(0, binding.STATIC_MAX_TASKSETS)
     _both(at_limit, binding.POLICY_GCAPS, 1024, 50)
+
+
+def test_a_call_allocates_and_frees_nothing():
+    """With the outputs in place beforehand, a call through the C-ABI must change neither the
+    driver's count of free device memory nor what torch's allocator holds."""
+    lib = binding.load_library()
+    batch = taskgen.WORKLOADS["sweep"].generate(3, 20_000)
+    ts = binding.DeviceTasksets.from_host(batch)
+    out_w = torch.zeros(ts.n_tasks, dtype=torch.int64, device="cuda")
+    out_s = torch.zeros(ts.n_tasksets, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call(policy):
+        rc = lib.gcaps_rta_batch_static(ctypes.byref(ts.c), ts.n_tasksets, policy, 1024, 50,
+                                        out_w.data_ptr(), out_s.data_ptr(), ctypes.c_void_p(stream))
+        assert rc == 0
+        torch.cuda.synchronize()
+
+    call(binding.POLICY_GCAPS)  # the first call on a device looks the scratch address up
+    free0, _ = torch.cuda.mem_get_info()
+    torch0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    call(binding.POLICY_RR)
+    call(binding.POLICY_GCAPS)
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_allocated() == torch0 and torch.cuda.memory_reserved() == reserved0
+    w_cpu, s_cpu, _ = rta.analyse(batch, binding.POLICY_GCAPS, 1024, 50)
+    assert np.array_equal(out_w.cpu().numpy(), w_cpu) and np.array_equal(out_s.cpu().numpy(), s_cpu)
