@@ -39,7 +39,7 @@ K_TERM, K_SETUP = 6, 16   # algorithmic integer lane-operations per interference
 # kernels launched by one gcaps_rta_batch call: 3 plan kernels, one analysis kernel for the bins
 # of up to 32 tasks and one each for the 64-, 96-, 128-, 192- and 256-task bins
 LAUNCHES_PER_CALL = 9        # three plan kernels + one kernel per group of size bins
-LAUNCHES_PER_SMALL_CALL = 7  # batches of up to 8,192 tasksets: one plan kernel
+LAUNCHES_PER_SMALL_CALL = 2  # batches of up to 8,192 tasksets: one plan kernel, one kernel for all bins
 # DRAM bytes (read + write) per taskset of the analysis kernel on the 'large' workload, from an
 # ncu capture of a 131,072-taskset launch (traffic grows in proportion to the tasksets of a
 # launch).  Only reported while the kernel source is the one the counters were taken from.
@@ -237,6 +237,9 @@ def main():
                          "gcaps_rta_sweep_batch call and once as one gcaps_rta_batch call per pair")
     ap.add_argument("--graph", action="store_true",
                     help="replay each call from a CUDA graph instead of enqueueing its launches again")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every rank analyses --tasksets tasksets of its own; strong: --tasksets "
+                         "tasksets in all, split over the ranks")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cpu-all-cores", action="store_true",
@@ -270,7 +273,12 @@ def main():
     binding.load_library()
 
     per_gpu = args.tasksets or min(workload.n_tasksets, MAX_TASKSETS_PER_GPU)
-    first, count = sharding.weak_shard(rank, per_gpu)
+    if args.scaling == "strong":   # a fixed job split over the ranks
+        first, count = sharding.strong_shard(rank, world, per_gpu)
+        total_count = per_gpu
+    else:                          # every rank analyses its own per_gpu tasksets
+        first, count = sharding.weak_shard(rank, per_gpu)
+        total_count = world * count
     pinned = []
 
     def alloc(n):
@@ -414,9 +422,9 @@ def main():
     sched_frac = float((flags == 1).float().mean().item()) if count else 0.0
     total_ms = sharding.reduce_scalars([total_ms], "max", dev)[0]
     ms_per_step = total_ms / args.steps
-    value = world * count / (ms_per_step * 1e-3)
+    value = total_count / (ms_per_step * 1e-3)
     if args.mode == "sweep":  # taskset analyses per second of the fused call alone
-        value = world * count * len(pairs) / (per_policy_ms[0] * 1e-3)
+        value = total_count * len(pairs) / (per_policy_ms[0] * 1e-3)
 
     # ---- beside the headline: the busy-waiting analyses, planning on its own, the integer peak --
     def mean_ms(fn, n):
@@ -472,7 +480,7 @@ def main():
         barrier()
         dt = time.perf_counter() - t0
         dt = sharding.reduce_scalars([dt], "max", dev)[0]
-        e2e = {"value": world * count * args.e2e_steps / dt, "unit": UNIT,
+        e2e = {"value": total_count * args.e2e_steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": batch.input_bytes(),
                "d2h_bytes_per_step": len(host_policies) * batch.output_bytes(),
                "steps": args.e2e_steps, "ms_per_step": 1e3 * dt / args.e2e_steps,
@@ -571,7 +579,7 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "scaling": args.scaling, "vs_baseline": None, "dtype": "int64", "data": "synthetic",
             "config": {"workload": workload.name, "note": workload.note, "tasksets_per_gpu": count,
                        "tasks": ts.n_tasks, "policies": names, "mode": "self-suspension",
                        "timeslice_us": L, "overhead_us": ovh,

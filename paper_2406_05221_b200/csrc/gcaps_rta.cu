@@ -39,6 +39,13 @@
 
 using namespace gcaps_detail;
 
+#ifndef GCAPS_PREFETCH_AHEAD
+#define GCAPS_PREFETCH_AHEAD 0
+#endif
+#ifndef GCAPS_FIRST_RANKS
+#define GCAPS_FIRST_RANKS 1
+#endif
+
 namespace {
 
 // ---------------------------------------------------------------------------------------------
@@ -464,6 +471,220 @@ __device__ __forceinline__ void prefix_step(const i64 *__restrict__ X0, const i6
   }
 }
 
+// Range check of segment slices without running sums: `bad` collects whether a wanted element lies
+// outside [0, 2^26), and the elements, narrowed to 32 bits, go to shared memory as they are
+// (D[w] = element w - par; same loads and store pattern as prefix_step).  NB blocks of 128
+// elements per array in flight together (TWO: two arrays that share their offsets).
+template <int NB, bool TWO>
+__device__ __forceinline__ void check_slices(const i64 *__restrict__ X0, const i64 *__restrict__ X1, int N,
+                                             int par0, int par1, bool inside, const i64 *lo0,
+                                             const i64 *hi0, const i64 *lo1, const i64 *hi1, u32 *D0,
+                                             u32 *D1, int lane, u32 &bad) {
+  for (int e0 = 0; e0 < N + (par0 > par1 ? par0 : par1); e0 += 128 * NB) {
+    Quad q0[NB], q1[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      if (inside) {
+        load_quad_inside(X0, e0 + 128 * b + 4 * lane - par0, N, q0[b]);
+        if (TWO) load_quad_inside(X1, e0 + 128 * b + 4 * lane - par1, N, q1[b]);
+      } else {
+        q0[b] = load_quad_edge(X0, e0 + 128 * b + 4 * lane - par0, N, lo0, hi0);
+        if (TWO) q1[b] = load_quad_edge(X1, e0 + 128 * b + 4 * lane - par1, N, lo1, hi1);
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      if (e0 + 128 * b < N + 1) {
+        u32 x[4];
+        narrow_quad(q0[b], e0 + 128 * b + 4 * lane - par0, N, x, bad);
+        *reinterpret_cast<uint4 *>(D0 + e0 + 128 * b + 4 * lane) =
+            make_uint4((u32)q0[b].v[0], (u32)q0[b].v[1], (u32)q0[b].v[2], (u32)q0[b].v[3]);
+        if (TWO) {
+          narrow_quad(q1[b], e0 + 128 * b + 4 * lane - par1, N, x, bad);
+          *reinterpret_cast<uint4 *>(D1 + e0 + 128 * b + 4 * lane) =
+              make_uint4((u32)q1[b].v[0], (u32)q1[b].v[1], (u32)q1[b].v[2], (u32)q1[b].v[3]);
+        }
+      }
+    }
+  }
+}
+
+// The first kFirstRanks tasks of the priority order, analysed before anything is summed for the
+// rest of the taskset (a warp per taskset).  Where tasksets are far from schedulable the first
+// deadline miss comes within a handful of ranks, and the per-task sums of all the other tasks
+// would never be used: here every segment value is still read and range-checked (a value outside
+// the 32-bit path's range sends the taskset to the exact path, as always), but sums are formed
+// only for these ranks: four lanes per rank add up the rank's own few segments, all ranks at once
+// (one trip to memory), and lane r then holds everything about rank r, as the task under analysis
+// and as an interferer of the ranks behind it.  The recurrence over these ranks needs registers
+// and warp collectives only.  Same arithmetic, same sequence of iterates, same sentinels as the
+// full pass.  `first8[r]` = (first, end) of rank r's CPU segments and of its GPU segments within
+// the taskset's slices; info[r] = (deadline, core, period, position).
+// Returns 1: the taskset is finished (a miss among these ranks, or no other real-time task), its
+// outputs are written; 0: all these ranks converged, the caller runs the full pass (which repeats
+// them); -1: a value does not fit the 32-bit path.
+constexpr int kFirstRanks = 8;
+template <int SLOTS, int MODE>
+__device__ __forceinline__ int first_ranks(const KParams &p, i64 t, i64 a, int n, const uint4 *info,
+                                           const uint4 *first8, u32 *Q0, u32 *Q1, int n_rt,
+                                           const int (&rank)[SLOTS], const int (&g0)[SLOTS],
+                                           const int (&g1)[SLOTS], const i64 *__restrict__ Xc,
+                                           const i64 *__restrict__ Xm, const i64 *__restrict__ Xe, int Nc,
+                                           int Ng, int parc, int parm, int pare, i64 cfirst, i64 gfirst,
+                                           int lane, bool literal) {
+  const int limit = n_rt < kFirstRanks ? n_rt : kFirstRanks;
+  // lanes 4r .. 4r+3 add up the segments of rank r
+  const int r4 = lane >> 2, sub = lane & 3;
+  uint4 seg = make_uint4(0u, 0u, 0u, 0u);
+  if (r4 < limit) seg = first8[r4];
+  u32 bad = 0, sum_c = 0, sum_m = 0, sum_e = 0, sum_s = 0;
+  // every segment value of the taskset must be in [0, 2^26); on the way the values stop over in
+  // shared memory, where the eight ranks find their own
+  check_slices<(SLOTS < 3 ? SLOTS : 3), false>(Xc, Xc, Nc, parc, parc, slice_is_inside(cfirst, Nc, parc, p.n_csegs),
+                                               p.cseg_wcet, p.cseg_wcet + p.n_csegs, p.cseg_wcet, p.cseg_wcet,
+                                               Q0, Q0, lane, bad);
+  __syncwarp();
+  for (int j = (int)seg.x + parc + sub; j < (int)seg.y + parc; j += 4) sum_c += Q0[j];
+  __syncwarp();
+  check_slices<2, true>(Xm, Xe, Ng, parm, pare,
+                        slice_is_inside(gfirst, Ng, parm, p.n_gsegs) && slice_is_inside(gfirst, Ng, pare, p.n_gsegs),
+                        p.gseg_misc, p.gseg_misc + p.n_gsegs, p.gseg_exec, p.gseg_exec + p.n_gsegs, Q1, Q0,
+                        lane, bad);
+  __syncwarp();
+  for (int j = (int)seg.z + sub; j < (int)seg.w; j += 4) {
+    sum_m += Q1[j + parm];
+    const u32 e = Q0[j + pare] & (kFastLimit - 1);  // (checked above; keeps the division exact)
+    sum_e += e;
+    if (MODE >= 2) {  // Eq. 3: slices of the pure GPU part
+      if (p.l_mode == 0) sum_s += __umulhi(e + (u32)p.L - 1u, p.l_magic) >> p.l_shift;
+      else if (p.l_mode == 1) sum_s += e;
+      else sum_s += e > 0 ? 1u : 0u;
+    }
+  }
+  int n_gpu = 0;  // N_g
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) n_gpu += __popc(__ballot_sync(kFull, g1[s] > g0[s]));
+#pragma unroll
+  for (int d = 1; d <= 2; d <<= 1) {
+    sum_c += __shfl_xor_sync(kFull, sum_c, d), sum_m += __shfl_xor_sync(kFull, sum_m, d);
+    sum_e += __shfl_xor_sync(kFull, sum_e, d);
+    if (MODE >= 2) sum_s += __shfl_xor_sync(kFull, sum_s, d);
+  }
+  // lane r takes rank r from lane 4r (a task has fewer than 64 segments of a kind, every value is
+  // below 2^26: no overflow)
+  const int src = (4 * lane) & 31;
+  sum_c = __shfl_sync(kFull, sum_c, src), sum_m = __shfl_sync(kFull, sum_m, src);
+  sum_e = __shfl_sync(kFull, sum_e, src);
+  if (MODE >= 2) sum_s = __shfl_sync(kFull, sum_s, src);
+  const u32 eta_r = __shfl_sync(kFull, seg.w - seg.z, src);
+  const bool mine = lane < limit;
+  const uint4 f = mine ? info[lane] : make_uint4(1u, 0xffffffffu, 2u, 0u);  // deadline, core, period, position
+  const u32 ovh = (u32)p.ovh;  // below 2^20 on this path
+  const u32 D_r = f.x, core_r = f.y, Tm1 = f.z - 1, A_r = sum_c + sum_m, Ge_r = sum_e;
+  const bool gpu_r = eta_r > 0;
+  u32 S_r, base_r;
+  if (MODE < 2) {
+    S_r = 2 * ovh * eta_r;                               // eta < 64: below 2^27
+    base_r = A_r + Ge_r + S_r + (eta_r + 1) * ovh;       // C_i + G*_i + B^C_i, below 2^29
+    if (mine) bad |= S_r >> 26;
+  } else {
+    const u64 lt = (u64)p.L + ovh;                       // <= 2^41
+    u64 B = sum_s == 0 ? 0 : (lt >= kFastClamp ? kFastClamp : lt * (u64)sum_s);
+    if (B > kFastClamp) B = kFastClamp;
+    S_r = (u32)B;
+    const u64 b64 = (u64)A_r + Ge_r + (gpu_r ? B * (u64)(n_gpu - 1) : 0);  // Lemma 1
+    base_r = b64 > (u64)(2 * kFastClamp) ? 2 * kFastClamp : (u32)b64;
+  }
+  base_r = base_r > 2 * kFastClamp ? 2 * kFastClamp : base_r;
+  if (mine) bad |= (sum_c | sum_m | A_r | Ge_r) >> 26;
+  if (__any_sync(kFull, bad != 0)) return -1;
+  u32 magic, shift;
+  make_reciprocal(f.z, magic, shift);
+  // what rank r contributes as an interferer (the jitters follow when it has converged)
+  u32 Wa, Wb;
+  if (MODE == 0) {
+    Wa = A_r + (gpu_r ? S_r : 0u);    // Lemma 15: C_h, or C_h + G^{m*}_h
+    Wb = gpu_r ? Ge_r + S_r : 0u;     // Lemma 13, other cores: G^{e*}_h
+  } else if (MODE == 1) {
+    Wa = A_r;                         // Lemma 12
+    Wb = gpu_r ? Ge_r + S_r : 0u;     // Lemmas 10, 11: G^{e*}_h
+  } else {
+    Wa = A_r;                         // Lemmas 5, 7
+    Wb = gpu_r ? S_r : 0u;            // Lemma 4: (L+theta) * slices
+  }
+  u32 Jc = Tm1, Jg = Tm1;
+  // ---- the recurrence of Eq. 1 over these ranks -----------------------------------------------------
+  int verdict = 0, pos = 0;
+  for (; pos < limit; ++pos) {
+    const u32 Di = __shfl_sync(kFull, D_r, pos), core_i = __shfl_sync(kFull, core_r, pos);
+    const u32 base_i = __shfl_sync(kFull, base_r, pos);
+    const bool gi = __shfl_sync(kFull, (int)gpu_r, pos) != 0;
+    const bool act = lane < pos, same = core_r == core_i;
+    u32 j1, w1, w2 = 0;
+    if (MODE == 0) {
+      w1 = same ? Wa : (gi ? Wb : 0u);            // Lemma 15 / Lemma 13 (other cores)
+      j1 = same ? Jc : Jg;
+      w2 = (same && gi && gpu_r) ? Ge_r : 0u;     // Lemma 13 (same core), jitter J^g
+    } else if (MODE == 1) {
+      w1 = same ? Wa + ((gi || !literal) ? Wb : 0u) : Wb;  // Lemmas 12+10 / 10, 11
+      j1 = same ? Tm1 : Jg;
+    } else if (MODE == 2) {
+      w1 = same ? Wa : 0u;                        // Lemma 7
+      j1 = Jc;
+    } else {
+      // Lemma 4: N_g - |{h in hpp(i): GPU-using}| + 1
+      const u32 nu = (u32)(n_gpu - __popc(__ballot_sync(kFull, act && same && gpu_r)) + 1);
+      const u64 w = (u64)Wa + (u64)Wb * nu;       // Lemmas 5 and 4
+      w1 = same ? (w > kFastClamp ? kFastClamp : (u32)w) : 0u;
+      j1 = Tm1;
+    }
+    if (!act) w1 = 0, w2 = 0;
+    u32 R = base_i;
+    int sweeps = 0;
+    for (;;) {
+      if (R > Di) {
+        verdict = GCAPS_WCRT_MISS;
+        break;
+      }
+      if (sweeps >= (int)GCAPS_RTA_ITER_CAP) {
+        verdict = GCAPS_WCRT_ITER_LIMIT;
+        break;
+      }
+      sweeps += 1;
+      u32 next = base_i;
+      if (pos > 0) {
+        u64 acc = (u64)(__umulhi(R + j1, magic) >> shift) * w1;
+        if (MODE == 0) acc += (u64)(__umulhi(R + Jg, magic) >> shift) * w2;
+        const u32 part = acc > (u64)kFastClamp ? kFastClamp : (u32)acc;
+        next += __reduce_add_sync(kFull, part);
+      }
+      if (next == R) break;
+      R = next;
+    }
+    if (verdict != 0) break;
+    // publish: R_i goes out; lane `pos` forms the jitters J^c = R - (C+G^m), J^g = R - G^e (a
+    // CPU-only task has no J^c unless the printed form of Lemma 7 is asked for)
+    if (lane == pos) {
+      if (p.out_wcrt) p.out_wcrt[a + f.w] = (i64)R;
+      if (MODE == 0 ? gpu_r : (MODE == 2 ? (gpu_r || literal) : false)) Jc = R - A_r + Tm1;
+      Jg = R - Ge_r + Tm1;
+    }
+  }
+  if (verdict == 0 && limit < n_rt) return 0;  // undecided: the full pass takes over
+  const int n_done = pos;  // ranks that converged (= n_rt without a verdict)
+  if (p.out_wcrt) {
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const int r = rank[s];
+      if (lane + 32 * s < n && r >= n_done)
+        p.out_wcrt[a + lane + 32 * s] = r >= n_rt ? (i64)GCAPS_WCRT_BEST_EFFORT
+                                                  : (r == n_done ? (i64)verdict : (i64)GCAPS_WCRT_SKIPPED);
+    }
+  }
+  if (lane == 0) p.out_sched[t] = verdict == 0 ? GCAPS_SCHED_YES : GCAPS_SCHED_NO;
+  return 1;
+}
+
 // An analysis mode known at compile time (converts to int like a run-time mode does).
 template <int V>
 struct ModeTag {
@@ -486,9 +707,16 @@ struct ModeTag {
 // q * sw->block_stride + sw->block_of_mode[m] (out_wcrt + block * n_tasks, skipped when out_wcrt
 // is null; out_sched + block * n_tasksets).  Without SWEEP, MASK has one bit and the analysis
 // takes its constants and outputs from `p`.
-template <int LPT, int SLOTS, int MASK, bool SWEEP = false>
-__device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane,
-                                             unsigned int gmask, const SweepArgs *sw = nullptr) {
+//
+// Returns kFastDone (outputs written), kFastDeclined (nothing written that matters: the caller runs
+// the exact path) or, with FIRST_ONLY, kFastUndecided.  FIRST_ONLY (one analysis, a warp per
+// taskset): only the first ranks of the priority order are analysed (first_ranks below); if they
+// all converge and more ranks follow, nothing is decided and the caller runs the full pass.
+constexpr int kFastDeclined = 0, kFastDone = 1, kFastUndecided = 2;
+template <int LPT, int SLOTS, int MASK, bool SWEEP = false, bool FIRST_ONLY = false>
+__device__ __forceinline__ int analyse_fast(const KParams &p, i64 t, i64 a, int n, u32 *buf, int lane,
+                                            unsigned int gmask, const SweepArgs *sw = nullptr) {
+  static_assert(!FIRST_ONLY || (LPT == 32 && !SWEEP), "the first ranks' own pass: a warp per taskset");
   typedef FastLayout<LPT, SLOTS> Lay;
   constexpr int kLog = LPT == 32 ? 5 : LPT == 16 ? 4 : 3;  // log2 of the lanes per taskset
   constexpr int MAXN = Lay::MAXN, CAP = Lay::CAP;
@@ -497,7 +725,11 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   // in one step where two need a second, mostly empty one (80-task tasksets: -4 % for a GCAPS
   // kernel; the RR kernels, which carry the slice sums too, lose as much to the registers it takes)
   constexpr int BC = SLOTS <= 2 ? SLOTS : ((SLOTS == 3 && (MASK & 12) == 0 && !SWEEP) ? 3 : 2);
+#ifdef GCAPS_BG2
+  constexpr int BG = (SLOTS == 3 && (MASK & 12) == 0 && !SWEEP) ? 2 : 1;
+#else
   constexpr int BG = 1;
+#endif
   constexpr bool kAnyGcaps = (MASK & 3) != 0;
   constexpr bool kMulti = (MASK & (MASK - 1)) != 0;
   static_assert(!kMulti || SWEEP, "several analyses per taskset use the sweep loop");
@@ -526,7 +758,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     const i64 Nc64 = cend - cfirst, Ng64 = gend - gfirst;
     if (cfirst < 0 || Nc64 < 0 || cend > p.n_csegs || Nc64 >= CAP || gfirst < 0 || Ng64 < 0 ||
         gend > p.n_gsegs || Ng64 >= CAP)
-      return false;
+      return kFastDeclined;
     Nc = (int)Nc64, Ng = (int)Ng64;
     u32 high = 0;  // any set bit: some value does not fit the 32-bit path
     u32 D[SLOTS], core[SLOTS];
@@ -549,7 +781,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       ok &= T[s] - 2u < kFastLimit - 2u && (!v || (D[s] - 1u < T[s] && (int)core[s] >= 0)) &&
             (u32)c0[s] <= (u32)Nc && (u32)g0[s] <= (u32)Ng;
     }
-    if (__any_sync(gmask, high != 0 || !ok)) return false;  // (a wide priority also lands here)
+    if (__any_sync(gmask, high != 0 || !ok)) return kFastDeclined;  // (a wide priority also lands here)
     // order: rank by (priority desc, position asc)
     int m = prio[0];
 #pragma unroll
@@ -600,11 +832,16 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       }
       if (lane == 0) Q0[-2] = (u32)n_rt;
     }
-    // what every lane must know about the task of a given rank (base and GPU flag follow)
+    // what every lane must know about the task of a given rank (base and GPU flag follow; the
+    // first ranks' own pass keeps the period and the position there instead)
 #pragma unroll
-    for (int s = 0; s < SLOTS; ++s)
-      if (lane + LPT * s < n)
-        *reinterpret_cast<uint2 *>(&info[rank[s]]) = make_uint2(D[s], core[s]);
+    for (int s = 0; s < SLOTS; ++s) {
+      if constexpr (FIRST_ONLY) {
+        if (rank[s] < kFirstRanks) info[rank[s]] = make_uint4(D[s], core[s], T[s], (u32)(lane + LPT * s));
+      } else {
+        if (lane + LPT * s < n) *reinterpret_cast<uint2 *>(&info[rank[s]]) = make_uint2(D[s], core[s]);
+      }
+    }
   }
   // end offsets: the next task's start (positions beyond n hold the total)
   int c1[SLOTS], g1[SLOTS];
@@ -617,7 +854,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
     g1[s] = lane == LPT - 1 ? gh : gn;
     ok &= (u32)(c1[s] - c0[s]) < 64u && (u32)(g1[s] - g0[s]) < 64u;
   }
-  if (!__all_sync(gmask, ok)) return false;
+  if (!__all_sync(gmask, ok)) return kFastDeclined;
 
   // ---- aggregate: running sums of the segment arrays; per-task sums are differences --------
   u32 A[SLOTS], Ge[SLOTS], S[SLOTS];  // C+G^m, G^e, and 2*eps*eta (GCAPS) or (L+theta)*slices (RR)
@@ -626,6 +863,18 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
   const i64 *__restrict__ Xm = p.gseg_misc + gfirst, *__restrict__ Xe = p.gseg_exec + gfirst;
   const int parc = (int)(((uintptr_t)Xc >> 3) & 1), parm = (int)(((uintptr_t)Xm >> 3) & 1);
   const int pare = (int)(((uintptr_t)Xe >> 3) & 1);
+  if constexpr (FIRST_ONLY) {
+    constexpr int MODE = (MASK & 1) ? 0 : (MASK & 2) ? 1 : (MASK & 4) ? 2 : 3;
+    uint4 *first8 = info + kFirstRanks;  // (only the first ranks' rows of `info` are used here)
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s)
+      if (rank[s] < kFirstRanks) first8[rank[s]] = make_uint4((u32)c0[s], (u32)c1[s], (u32)g0[s], (u32)g1[s]);
+    __syncwarp(gmask);
+    const int r = first_ranks<SLOTS, MODE>(p, t, a, n, info, first8, Q0, Q1, (int)Q0[-2], rank, g0, g1, Xc, Xm, Xe,
+                                           Nc, Ng, parc, parm, pare, cfirst, gfirst, lane, literal);
+    __syncwarp(gmask);
+    return r > 0 ? kFastDone : (r == 0 ? kFastUndecided : kFastDeclined);
+  }
   if (lane == 0) Q0[-1] = 0, Q1[-1] = 0;
   {  // CPU segments -> Q0
     const bool inside = slice_is_inside(cfirst, Nc, parc, p.n_csegs);
@@ -667,7 +916,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) bad |= (2 * ovh_max * eta[s]) >> 26;
   }
-  if (__any_sync(gmask, bad != 0)) return false;
+  if (__any_sync(gmask, bad != 0)) return kFastDeclined;
   const int n_rt_all = (int)Q0[-2];  // real-time tasks: the ranks that are analysed
   uint4 *xch = reinterpret_cast<uint4 *>(Q0);  // by rank: T, C+G^m, G^e, S  (Q0 is dead by now)
 
@@ -984,7 +1233,7 @@ __device__ __forceinline__ bool analyse_fast(const KParams &p, i64 t, i64 a, int
       if ((MASK & 8) && (enabled & 8)) analyse_as(ModeTag<3>());
     }
   }
-  return true;
+  return kFastDone;
 }
 
 __device__ __forceinline__ void prefetch_l2(const void *ptr) {
@@ -1060,6 +1309,7 @@ __device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf
   };
   static_assert(MAXN <= 256 && Lay::CAP <= 2048, "fields of Ahead::packed");
 
+  int undecided_run = 0, tried_since = 0;  // (the first ranks' own pass, see below)
   unsigned int first = 0;
   if (lane32 == 0) first = atomicAdd(&p.hdr->next[bin], (unsigned int)chunk);
   first = __shfl_sync(kFull, first, 0);
@@ -1089,9 +1339,50 @@ __device__ __forceinline__ void run_bin(const KParams &p, int bin, u32 *warp_buf
         for (int e = 16 * lane; e < nc; e += 16 * LPT) prefetch_l2(p.cseg_wcet + me.c_lo + e);
         for (int e = 16 * lane; e < ng; e += 16 * LPT)
           prefetch_l2(p.gseg_misc + me.g_lo + e), prefetch_l2(p.gseg_exec + me.g_lo + e);
+#if GCAPS_PREFETCH_AHEAD
+        // the per-task arrays of the group's next taskset of this pull start their way into L2 while
+        // this one is analysed (one 128-byte line per lane and array; a taskset has at most 256
+        // tasks, i.e. 17 lines of an array)
+        if (mine + G < in_chunk) {
+          const Ahead nx = cur[mine + G];
+          const int nn = (int)(nx.packed & 0x1ffu);
+          if ((nx.packed >> 31) != 0 && lane < 17) {
+            const i64 *arrays[6] = {p.period, p.deadline, p.priority, p.core, p.cseg_off, p.gseg_off};
+#pragma unroll
+            for (int k = 0; k < 6; ++k) {
+              const uintptr_t lo = reinterpret_cast<uintptr_t>(arrays[k] + nx.a);
+              const uintptr_t line = (lo & ~(uintptr_t)127) + 128u * (unsigned)lane;
+              if (line < lo + 8u * (unsigned)(nn + (k >= 4 ? 1 : 0))) prefetch_l2(reinterpret_cast<const void *>(line));
+            }
+          }
+#if GCAPS_PREFETCH_AHEAD > 1
+          const int nnc = (int)((nx.packed >> 9) & 0x7ffu), nng = (int)((nx.packed >> 20) & 0x7ffu);
+          for (int e = 16 * lane; e < nnc; e += 16 * LPT) prefetch_l2(p.cseg_wcet + nx.c_lo + e);
+          for (int e = 16 * lane; e < nng; e += 16 * LPT)
+            prefetch_l2(p.gseg_misc + nx.g_lo + e), prefetch_l2(p.gseg_exec + nx.g_lo + e);
+#endif
+        }
+#endif
         bool done = false;
-        if (fast_call && (me.packed >> 31) != 0)
-          done = analyse_fast<LPT, SLOTS, MASK, SWEEP>(p, t, me.a, n, buf, lane, gmask, sw);
+        if (fast_call && (me.packed >> 31) != 0) {
+          int how = kFastUndecided;
+          if constexpr (LPT == 32 && !SWEEP && (MASK & 12) != 0 && GCAPS_FIRST_RANKS != 0) {
+            // Far from schedulable, a taskset ends with a miss among its first ranks; nearly
+            // schedulable, looking at them first is wasted.  Tasksets of a batch tend to be alike:
+            // after four undecided ones in a row only every sixteenth taskset is tried that way.
+            // (Round robin only: with tens of GPU-using tasks taking turns on the GPU the first or
+            // second rank already misses, and the pass pays; under GCAPS the first miss comes a few
+            // ranks later and the pass was measured slower than the full one.)
+            if (undecided_run < 4 || (tried_since & 15) == 0) {
+              how = analyse_fast<LPT, SLOTS, MASK, false, true>(p, t, me.a, n, buf, lane, gmask);
+              undecided_run = how == kFastUndecided ? undecided_run + 1 : 0;
+              __syncwarp(gmask);
+            }
+            tried_since += 1;
+          }
+          if (how == kFastUndecided) how = analyse_fast<LPT, SLOTS, MASK, SWEEP>(p, t, me.a, n, buf, lane, gmask, sw);
+          done = how == kFastDone;
+        }
         __syncwarp(gmask);
         if (!done && !SWEEP) {
           // the exact path reads task_off again and validates everything itself
@@ -1158,6 +1449,28 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kern
   u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kWarpWords;
   Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kWarpWords - kAheadWords);
   run_bin<32, SLOTS, 1 << MODE>(p, bin, warp_buf, ahead);
+  wait_for_previous_grid();
+}
+
+// All nine bins in one launch, for batches so small (at most kPlanSmall tasksets) that the
+// launches of a call cost more than its work: a call is then the one-block plan kernel and this.
+// Registers and shared memory are those of the largest bin, which such a batch can afford.
+constexpr int kAnyWarpWords = cmax(kSmallWarpWords, bin_warp_words<32, 8>() + kAheadWords);
+template <int MODE>
+__global__ void __launch_bounds__(kBlockThreads, 2) rta_any_kernel(KParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  let_dependents_start();
+  u32 *warp_buf = reinterpret_cast<u32 *>(smem_raw) + (threadIdx.x >> 5) * kAnyWarpWords;
+  Ahead *ahead = reinterpret_cast<Ahead *>(warp_buf + kAnyWarpWords - kAheadWords);
+  run_bin<32, 8, 1 << MODE>(p, 8, warp_buf, ahead);
+  run_bin<32, 6, 1 << MODE>(p, 7, warp_buf, ahead);
+  run_bin<32, 4, 1 << MODE>(p, 6, warp_buf, ahead);
+  run_bin<32, 3, 1 << MODE>(p, 5, warp_buf, ahead);
+  run_bin<32, 2, 1 << MODE>(p, 4, warp_buf, ahead);
+  run_bin<16, 2, 1 << MODE>(p, 3, warp_buf, ahead);
+  run_bin<8, 3, 1 << MODE>(p, 2, warp_buf, ahead);
+  run_bin<8, 2, 1 << MODE>(p, 1, warp_buf, ahead);
+  run_bin<8, 1, 1 << MODE>(p, 0, warp_buf, ahead);
   wait_for_previous_grid();
 }
 
@@ -1350,6 +1663,11 @@ cudaError_t launch_big(const KParams &p, int bin, int sm_count, cudaStream_t st)
 template <int MODE>
 cudaError_t launch_all_bins(const KParams &p, int sm_count, cudaStream_t st) {
   constexpr int kWarps = kBlockThreads / 32;
+  if (p.n_tasksets <= kPlanSmall) {  // one launch for every bin
+    static int any_blocks_per_sm[64] = {0};
+    return launch_persistent(rta_any_kernel<MODE>, any_blocks_per_sm, sizeof(u32) * kAnyWarpWords * kWarps,
+                             (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p);
+  }
   static int blocks_per_sm[64] = {0};
   const size_t smem = sizeof(u32) * kSmallWarpWords * kWarps;
   cudaError_t e = launch_persistent(rta_small_kernel<MODE>, blocks_per_sm, smem,
