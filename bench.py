@@ -44,10 +44,10 @@ LAUNCHES_PER_SMALL_CALL = 2  # batches of up to 8,192 tasksets: one plan kernel,
 # ncu capture of a 131,072-taskset launch (traffic grows in proportion to the tasksets of a
 # launch).  Only reported while the kernel source is the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "992c86b02973be248905087f74519284979b90198204ab7a2bd867e3b67426d8",
+    "source_sha256": "192008cb141a5c691eced2e88153bc462b1b860986f152d05d382bbdf6a8b9fa",
     "workload": "large",
-    "bytes_per_taskset": {"gcaps": (1248971000 + 84039424) / 131072.0,
-                          "rr": (1247874000 + 84161792) / 131072.0},
+    "bytes_per_taskset": {"gcaps": (1248476000 + 84340736) / 131072.0,
+                          "rr": (1258324000 + 95665152) / 131072.0},
 }
 
 
