@@ -81,6 +81,17 @@ def test_workload_samples(name, count):
             assert s.max() == 1  # the easy end of the sweep has schedulable tasksets
 
 
+def test_converging_large_tasksets():
+    """Tasksets of 80 tasks that are schedulable under GCAPS: the recurrence runs for every task
+    (two to three ranks per lane), every bound is a converged value."""
+    w = taskgen.WORKLOADS["large_light"]
+    b = w.generate(5, 1200)
+    for policy in MODES4:
+        wc, s = assert_parity(b, policy, w.timeslice_us, w.overhead_us, "large_light")
+        if policy == 0:
+            assert s.min() == 1 and wc.min() > 0
+
+
 def test_rr_driver_model_grid():
     w = taskgen.WORKLOADS["rr_model"]
     b = w.generate(0, 1500)
