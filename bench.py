@@ -44,7 +44,7 @@ LAUNCHES_PER_SMALL_CALL = 2  # batches of up to 8,192 tasksets: one plan kernel,
 # ncu capture of a 131,072-taskset launch (traffic grows in proportion to the tasksets of a
 # launch).  Only reported while the kernel source is the one the counters were taken from.
 CAPTURED_TRAFFIC = {
-    "source_sha256": "192008cb141a5c691eced2e88153bc462b1b860986f152d05d382bbdf6a8b9fa",
+    "source_sha256": "9fc3a243eb31c6fb7c4e05766b9dc8d537e4e9f0aa84ad3911c2ef4eedab4396",
     "workload": "large",
     "bytes_per_taskset": {"gcaps": (1248476000 + 84340736) / 131072.0,
                           "rr": (1258324000 + 95665152) / 131072.0},

@@ -7,14 +7,15 @@ import sys
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CUDA_SRC = os.path.join(_HERE, "csrc", "gcaps_rta.cu")
-CUDA_SRCS = [CUDA_SRC, os.path.join(_HERE, "csrc", "gcaps_gpu_priority.cu"),
+CUDA_SRCS = [CUDA_SRC, os.path.join(_HERE, "csrc", "gcaps_rta_any.cu"),
+             os.path.join(_HERE, "csrc", "gcaps_gpu_priority.cu"),
              os.path.join(_HERE, "csrc", "gcaps_igen.cu"), os.path.join(_HERE, "csrc", "gcaps_diag.cu")]
 CUDA_DEPS = CUDA_SRCS + [os.path.join(_HERE, "csrc", "rta_common.cuh"), os.path.join(_HERE, "csrc", "igen.h")]
 CUDA_LIB = os.path.join(_HERE, "libgcaps_rta.so")
 HEADER = os.path.join(os.path.dirname(_HERE), "include", "gcaps_rta.h")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-shared", "-Xcompiler", "-fPIC", "--threads", "3"]
+              "-shared", "-Xcompiler", "-fPIC", "--threads", "5"]
 
 
 def _nvcc() -> str:

@@ -1455,6 +1455,7 @@ __global__ void __launch_bounds__(kBlockThreads, min_blocks(SLOTS)) rta_big_kern
 // All nine bins in one launch, for batches so small (at most kPlanSmall tasksets) that the
 // launches of a call cost more than its work: a call is then the one-block plan kernel and this.
 // Registers and shared memory are those of the largest bin, which such a batch can afford.
+#ifdef GCAPS_RTA_ANY_TU
 constexpr int kAnyWarpWords = cmax(kSmallWarpWords, bin_warp_words<32, 8>() + kAheadWords);
 template <int MODE>
 __global__ void __launch_bounds__(kBlockThreads, 2) rta_any_kernel(KParams p) {
@@ -1473,6 +1474,7 @@ __global__ void __launch_bounds__(kBlockThreads, 2) rta_any_kernel(KParams p) {
   run_bin<8, 1, 1 << MODE>(p, 0, warp_buf, ahead);
   wait_for_previous_grid();
 }
+#endif  // GCAPS_RTA_ANY_TU
 
 // The same launches for a fused sweep: every taskset is read once and analysed under all the
 // (timeslice, overhead) pairs of `sw`.
@@ -1540,6 +1542,29 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 size_t plan_blocks(int64_t n_tasksets) { return (size_t)((n_tasksets + kPlanItems - 1) / kPlanItems); }
 
 }  // namespace
+
+#ifdef GCAPS_RTA_ANY_TU
+// This file compiled as gcaps_rta_any.cu: only the all-bins kernels and their launcher (they
+// hold one copy of the device code per size bin and analysis, and compiling them beside the
+// other kernels rather than after them shortens the build).
+namespace gcaps_detail {
+
+cudaError_t launch_any_bins(int mode, const KParams &p, int sm_count, cudaStream_t st) {
+  constexpr int kWarps = kBlockThreads / 32;
+  static int blocks_per_sm[4][64] = {{0}};
+  const size_t smem = sizeof(u32) * kAnyWarpWords * kWarps;
+  const long long want = (p.n_tasksets + kWarps - 1) / kWarps;
+  switch (mode) {
+    case 0: return launch_persistent(rta_any_kernel<0>, blocks_per_sm[0], smem, want, sm_count, st, p);
+    case 1: return launch_persistent(rta_any_kernel<1>, blocks_per_sm[1], smem, want, sm_count, st, p);
+    case 2: return launch_persistent(rta_any_kernel<2>, blocks_per_sm[2], smem, want, sm_count, st, p);
+    case 3: return launch_persistent(rta_any_kernel<3>, blocks_per_sm[3], smem, want, sm_count, st, p);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace gcaps_detail
+#else
 
 // ---------------------------------------------------------------------------------------------
 // host side shared with the other translation units of the library
@@ -1663,11 +1688,7 @@ cudaError_t launch_big(const KParams &p, int bin, int sm_count, cudaStream_t st)
 template <int MODE>
 cudaError_t launch_all_bins(const KParams &p, int sm_count, cudaStream_t st) {
   constexpr int kWarps = kBlockThreads / 32;
-  if (p.n_tasksets <= kPlanSmall) {  // one launch for every bin
-    static int any_blocks_per_sm[64] = {0};
-    return launch_persistent(rta_any_kernel<MODE>, any_blocks_per_sm, sizeof(u32) * kAnyWarpWords * kWarps,
-                             (p.n_tasksets + kWarps - 1) / kWarps, sm_count, st, p);
-  }
+  if (p.n_tasksets <= kPlanSmall) return launch_any_bins(MODE, p, sm_count, st);  // one launch for every bin
   static int blocks_per_sm[64] = {0};
   const size_t smem = sizeof(u32) * kSmallWarpWords * kWarps;
   cudaError_t e = launch_persistent(rta_small_kernel<MODE>, blocks_per_sm, smem,
@@ -2137,3 +2158,4 @@ int gcaps_rta_last_cuda_error(void) { return g_last_cuda_error; }
 int gcaps_rta_version(void) { return GCAPS_RTA_VERSION; }
 
 }  // extern "C"
+#endif  // GCAPS_RTA_ANY_TU

@@ -230,6 +230,9 @@ void fill_params(KParams *p, const gcaps_tasksets_t *ts, int64_t n_tasksets, int
 // Points p at the plan areas of `workspace` and enqueues the three plan kernels (size bins, a
 // permutation of the taskset indices, zeroed work counters).  GCAPS_OK or GCAPS_ERR_WORKSPACE.
 int enqueue_plan(KParams &p, void *workspace, size_t workspace_bytes, cudaStream_t st);
+// One launch over all size bins for analysis `mode` (0 GCAPS self-suspension, 1 GCAPS
+// busy-waiting, 2 RR self-suspension, 3 RR busy-waiting); defined in gcaps_rta_any.cu.
+cudaError_t launch_any_bins(int mode, const KParams &p, int sm_count, cudaStream_t st);
 
 }  // namespace gcaps_detail
 #endif  // GCAPS_RTA_COMMON_CUH_
